@@ -1,0 +1,215 @@
+/*
+ * pdkv -- block-free transfer of paged KVCache between a prefill pool and a
+ * decode pool on one GPU (C ABI).
+ *
+ * The operations follow P/D-Serve, Sec. 3.5 "Block-free D2D KVCache Transfer":
+ * the sender organises a request's discrete KV blocks into one contiguous
+ * buffer ("Contiguous Buffer at Sender"), the bytes move as a whole, and the
+ * receiver restores discrete blocks from them ("RecvScatter at Receiver").
+ * Both sides manage HBM in fixed-size blocks (Sec. 2.3 "Block-fixed
+ * Management").  Here both pools live in the same GPU's memory, so a fused
+ * blocks-to-blocks call exists beside pack and unpack, and the block-by-block
+ * transfer the paper argues against (Sec. 2.3 "Unnecessary Controls") is kept
+ * as a timed baseline.
+ *
+ * Conventions
+ *   - Every function returns 0 (PDKV_OK) or a negative pdkv_status.  Nothing
+ *     throws, aborts or exits.  pdkv_strerror() names a status; after
+ *     PDKV_ERR_CUDA it also carries the CUDA error string of the calling thread.
+ *   - "device" pointers are CUDA device addresses on the pool's device; "host"
+ *     pointers are ordinary process memory.  The library borrows pools, buffers
+ *     and streams from the caller and never frees them.  It owns only a plan's
+ *     small device arrays (tile lists), freed by pdkv_plan_destroy().
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  pack / unpack / transfer only enqueue work: no allocation, no
+ *     host<->device copy, no synchronisation.
+ *   - Elements are opaque: `elem_bytes` bytes are moved bit for bit (NaN
+ *     payloads and -0 survive).
+ *
+ * Pool layouts (b = block id, tt = token slot inside the block)
+ *   PDKV_LAYOUT_BLOCK_MAJOR  [block][layer][K/V][token][head][dim]
+ *       elem = ((((b*L + l)*2 + c)*B + tt)*H + h)*D + d
+ *   PDKV_LAYOUT_LAYER_MAJOR  [layer][K/V][block][head][token][dim]
+ *       elem = ((((l*2 + c)*NB + b)*H + h)*B + tt)*D + d
+ *
+ * Contiguous buffer (Sec. 3.5: K and V of each layer "one after another";
+ * a layer's offset and length follow from prompt length, hidden size and
+ * precision): requests are concatenated in batch order without padding; inside
+ * request r the order is [layer][K/V][kept token][head][dim].  With n_r kept
+ * tokens, layer l of request r is the byte range
+ *       [ off_r + l*2*n_r*H*D*E ,  + 2*n_r*H*D*E ),
+ * where off_r is the exclusive prefix sum of 2*L*n_q*H*D*E over earlier
+ * requests q.  A layer range [layer_begin, layer_end) touches only those
+ * ranges, at the same offsets as a whole-model call.
+ *
+ * Skip mask: entry j of a request's decode table may be marked resident
+ * (shared prefix already on the decode side).  Token t is kept iff entry
+ * t / skip_granule_tokens is unmarked; marked blocks are neither packed nor
+ * written.  rank_r(t) is the number of kept tokens before t.
+ */
+#ifndef PDKV_H
+#define PDKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pdkv_pool pdkv_pool; /* opaque: geometry + borrowed device base */
+typedef struct pdkv_plan pdkv_plan; /* opaque: validated batch + device tile lists */
+
+enum pdkv_layout {
+    PDKV_LAYOUT_BLOCK_MAJOR = 0,
+    PDKV_LAYOUT_LAYER_MAJOR = 1
+};
+
+enum pdkv_status {
+    PDKV_OK = 0,
+    PDKV_ERR_INVALID_ARG = -1,      /* NULL, negative count, bad layer range, misaligned base */
+    PDKV_ERR_GEOMETRY = -2,         /* non-positive sizes; pools disagree on L/H/D/E */
+    PDKV_ERR_TABLE = -3,            /* block id out of range, table too short, duplicate decode block */
+    PDKV_ERR_BUFFER_TOO_SMALL = -4, /* contiguous buffer smaller than the plan needs */
+    PDKV_ERR_CUDA = -5,             /* a CUDA runtime call failed */
+    PDKV_ERR_DEVICE_BOUNDS = -6,    /* bounds-checked kernels refused an access (debug option) */
+    PDKV_ERR_NOMEM = -7             /* host allocation failed */
+};
+
+enum pdkv_op {
+    PDKV_OP_PACK = 0,
+    PDKV_OP_UNPACK = 1,
+    PDKV_OP_TRANSFER = 2
+};
+
+/* Geometry of one block-fixed pool (Sec. 2.3 "Block-fixed Management"). */
+typedef struct {
+    int32_t layout;       /* enum pdkv_layout */
+    int32_t num_layers;   /* L */
+    int32_t num_kv_heads; /* H */
+    int32_t head_dim;     /* D */
+    int32_t elem_bytes;   /* E: 1, 2, 4 or 8 */
+    int32_t block_tokens; /* B, any positive value */
+    int64_t num_blocks;   /* NB */
+} pdkv_pool_desc;
+
+/* One transfer batch.  All arrays are host memory, read only during
+ * pdkv_plan_create() (they are copied).  Tables are CSR: request r owns
+ * entries [off[r], off[r+1]); it needs at least ceil(seq_len[r] / B) of them
+ * and extra entries are ignored.  src_* may be NULL when the plan has no
+ * prefill pool, dst_tbl may be NULL when it has no decode pool; dst_tbl_off is
+ * still required when dst_skip is given, because the mask is parallel to the
+ * decode table. */
+typedef struct {
+    int32_t n_req;
+    const int32_t *seq_len;     /* [n_req] prompt tokens */
+    const int64_t *src_tbl_off; /* [n_req+1] */
+    const int32_t *src_tbl;     /* prefill block ids; duplicates allowed */
+    const int64_t *dst_tbl_off; /* [n_req+1] */
+    const int32_t *dst_tbl;     /* decode block ids; a used id may appear once */
+    const uint8_t *dst_skip;    /* parallel to dst_tbl; NULL = keep everything */
+} pdkv_batch_desc;
+
+/* Bytes the caller must allocate for a pool of this geometry (0 if invalid). */
+size_t pdkv_pool_bytes(const pdkv_pool_desc *desc);
+
+/* Wrap caller-owned device memory as a pool.  `dev_base` (device) must be
+ * 16-byte aligned and hold at least pdkv_pool_bytes() bytes on CUDA device
+ * `device`.  The pool keeps the pointer; it never frees or touches the memory.
+ * Errors: INVALID_ARG, GEOMETRY, NOMEM. */
+int pdkv_pool_create(const pdkv_pool_desc *desc, void *dev_base, size_t bytes,
+                     int device, pdkv_pool **out);
+int pdkv_pool_destroy(pdkv_pool *pool);
+
+/* Validate a batch against the pools and build the device-side tile lists --
+ * the single-GPU counterpart of the one low-cost meta exchange that precedes a
+ * transfer (Sec. 3.5).  `src` or `dst` may be NULL for a pack-only or
+ * unpack-only plan (not both).  `skip_granule_tokens` must equal the decode
+ * block size when `dst` is given; it is only free for pack-only plans (<= 0
+ * selects it from `dst`).  One small host->device copy is enqueued on `stream`
+ * and the call waits for it; later calls on other streams are therefore safe.
+ * Errors: INVALID_ARG, GEOMETRY, TABLE, CUDA, NOMEM; *out is NULL on error. */
+int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst,
+                     int32_t skip_granule_tokens, const pdkv_batch_desc *batch,
+                     void *stream, pdkv_plan **out);
+int pdkv_plan_destroy(pdkv_plan *plan);
+
+/* Size of the contiguous buffer in bytes and, optionally, the host array of
+ * n_req+1 request offsets off_r (owned by the plan, valid until destroy). */
+int pdkv_plan_buffer(const pdkv_plan *plan, size_t *total_bytes,
+                     const int64_t **req_off_bytes);
+
+/* Algorithmic traffic of one whole-model call of `op` (enum pdkv_op):
+ * payload bytes read, and payload plus zero-padding bytes written.  Tile
+ * metadata is not counted. */
+int pdkv_plan_traffic(const pdkv_plan *plan, int op, uint64_t *bytes_read,
+                      uint64_t *bytes_written);
+
+/* Sender side, Sec. 3.5 "Contiguous Buffer at Sender": gather every kept token
+ * of layers [layer_begin, layer_end) from the prefill pool into `buf` (device,
+ * 16-byte aligned, buf_bytes >= pdkv_plan_buffer()).  Bytes of `buf` outside
+ * the addressed layer ranges keep their value.
+ * Errors: INVALID_ARG, BUFFER_TOO_SMALL, CUDA. */
+int pdkv_pack(const pdkv_plan *plan, void *buf, size_t buf_bytes,
+              int layer_begin, int layer_end, void *stream);
+
+/* Receiver side, Sec. 3.5 "RecvScatter at Receiver": restore decode blocks of
+ * layers [layer_begin, layer_end) from `buf`, then zero the token slots past
+ * the prompt's end in each request's last decode block (unless that block is
+ * marked resident).  All other bytes of the decode pool are left untouched. */
+int pdkv_unpack(const pdkv_plan *plan, const void *buf, size_t buf_bytes,
+                int layer_begin, int layer_end, void *stream);
+
+/* Fused blocks-to-blocks: same decode pool image as pdkv_pack followed by
+ * pdkv_unpack, without materialising the buffer.  (No counterpart in the
+ * paper, whose two pools sit on different devices.) */
+int pdkv_transfer(const pdkv_plan *plan, int layer_begin, int layer_end, void *stream);
+
+/* Baseline: the block-by-block transfer of Sec. 2.3 ("transfer one by one"),
+ * one copy or one kernel launch per prefill block issued from a host loop.
+ * Same result as pdkv_transfer over all layers. */
+int pdkv_transfer_blockwise(const pdkv_plan *plan, void *stream);
+
+/* Number of GPU operations (kernel launches + memcpys) one call of `op`
+ * enqueues; op = 3 asks about pdkv_transfer_blockwise. */
+int pdkv_plan_launches(const pdkv_plan *plan, int op, int64_t *launches);
+
+/* One entry of a plan's tile list, for inspection and host-side tests: `ntok`
+ * consecutive kept tokens of one request lying inside one block on every paged
+ * side.  Offsets are bytes from the side's base for layer 0 / K; (l, c) adds
+ * (2*l + c) times the side's per-(l,c) stride, which for the contiguous buffer
+ * is n_kept*H*D*E.  src_off < 0 marks a zero-fill tile (tail slots). */
+typedef struct {
+    int64_t src_off;
+    int64_t dst_off;
+    int32_t ntok;
+    int32_t n_kept;
+} pdkv_tile;
+
+/* Host copy of the tile list of `op`, owned by the plan. */
+int pdkv_plan_tiles(const pdkv_plan *plan, int op, const pdkv_tile **tiles, int64_t *n_tiles);
+
+/* Synchronise `stream` and report the bounds-check word of the plan: PDKV_OK,
+ * PDKV_ERR_DEVICE_BOUNDS (an access was refused and skipped) or
+ * PDKV_ERR_CUDA.  Only meaningful with the "debug_bounds" option set. */
+int pdkv_plan_status(const pdkv_plan *plan, void *stream);
+
+/* Process-wide tunables, read when a plan is created or a call is launched:
+ *   "tile_bytes"     target bytes moved per tile (default 65536)
+ *   "ctas_per_sm"    persistent CTAs per SM (default 4)
+ *   "threads"        threads per CTA, multiple of 32 (default 512)
+ *   "lc_fastest"     1: consecutive work items walk layers of one tile (default 1)
+ *   "debug_bounds"   1: kernels range-check every access and skip bad ones
+ *   "variant"        0: register copy, 1: bulk async copy through shared memory
+ *   "dry_run"        1: pdkv_plan_create builds host-only plans (no CUDA call is
+ *                    made; the plan can be inspected but not launched)
+ * Unknown keys or out-of-range values give INVALID_ARG. */
+int pdkv_tune(const char *key, int64_t value);
+int pdkv_tune_get(const char *key, int64_t *value);
+
+const char *pdkv_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PDKV_H */

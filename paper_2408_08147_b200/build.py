@@ -1,0 +1,55 @@
+"""Build the C-ABI shared library (sm_100a) next to this file."""
+from __future__ import annotations
+
+import glob
+import os
+import shutil
+import subprocess
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_ROOT = os.path.dirname(_HERE)
+LIB_PATH = os.path.join(_HERE, "libpdkv.so")
+
+NVCC_FLAGS = [
+    "-gencode", "arch=compute_100a,code=sm_100a",
+    "-O3", "-std=c++17", "-lineinfo",
+    "-Xcompiler", "-fPIC,-Wall,-Wextra",
+    "-shared",
+]
+
+
+def sources() -> list[str]:
+    src = sorted(glob.glob(os.path.join(_HERE, "csrc", "*.cu")) +
+                 glob.glob(os.path.join(_HERE, "csrc", "*.cpp")))
+    return src
+
+
+def _stale() -> bool:
+    if not os.path.exists(LIB_PATH):
+        return True
+    t = os.path.getmtime(LIB_PATH)
+    deps = sources() + glob.glob(os.path.join(_HERE, "csrc", "*.h")) + \
+        glob.glob(os.path.join(_ROOT, "include", "*.h"))
+    return any(os.path.getmtime(d) > t for d in deps)
+
+
+def build_library(force: bool = False, verbose: bool = False) -> str:
+    """Compile every CUDA/C++ source into ``libpdkv.so`` with nvcc for sm_100a."""
+    if not force and not _stale():
+        return LIB_PATH
+    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+    tmp = LIB_PATH + f".{os.getpid()}.tmp"
+    cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(_ROOT, "include"),
+           "-I", os.path.join(_HERE, "csrc"), "-o", tmp, *sources()]
+    if verbose:
+        cmd.insert(1, "-Xptxas=-v")
+        print(" ".join(cmd))
+    subprocess.check_call(cmd)
+    os.replace(tmp, LIB_PATH)
+    return LIB_PATH
+
+
+if __name__ == "__main__":
+    import sys
+
+    print(build_library(force=True, verbose="-v" in sys.argv))

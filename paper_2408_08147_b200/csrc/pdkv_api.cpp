@@ -1,0 +1,638 @@
+// C-ABI entry points and the host planner: validates a batch against the two
+// pools, computes the contiguous buffer's per-request offsets (Sec. 3.5: a
+// layer's offset and length follow from prompt length, hidden size and
+// precision), cuts the batch into tiles and uploads the tile lists once.  This
+// is the single-GPU counterpart of the meta exchange that precedes a transfer.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "pdkv_internal.h"
+
+struct pdkv_pool {
+    pdkv_pool_desc d;
+    char *base;
+    size_t bytes;
+    int device;
+};
+
+namespace {
+
+using pdkv::Tile;
+
+struct BlockGroup {     // one prefill block's share of the fused transfer (baseline)
+    int32_t tile_begin, tile_end;
+    int64_t memcpy_src, memcpy_dst, memcpy_bytes;  // memcpy_bytes > 0: plain copy suffices
+};
+
+thread_local std::string g_cuda_msg;
+
+int cuda_fail(cudaError_t e, const char *what)
+{
+    g_cuda_msg = std::string("CUDA error in ") + what + ": " + cudaGetErrorString(e);
+    return PDKV_ERR_CUDA;
+}
+
+bool desc_ok(const pdkv_pool_desc *d)
+{
+    if (!d) return false;
+    if (d->layout != PDKV_LAYOUT_BLOCK_MAJOR && d->layout != PDKV_LAYOUT_LAYER_MAJOR) return false;
+    if (d->num_layers <= 0 || d->num_kv_heads <= 0 || d->head_dim <= 0 || d->block_tokens <= 0 ||
+        d->num_blocks <= 0)
+        return false;
+    if (d->elem_bytes != 1 && d->elem_bytes != 2 && d->elem_bytes != 4 && d->elem_bytes != 8)
+        return false;
+    // every byte offset must fit a signed 64-bit integer with room to spare
+    long double total = (long double)d->num_blocks * d->num_layers * 2.0L * d->block_tokens *
+                        d->num_kv_heads * d->head_dim * d->elem_bytes;
+    if (total > 4.0e18L) return false;
+    // a single (block, layer, K/V) strip must stay below 2^31 vectors of one byte
+    long double strip = (long double)d->block_tokens * d->num_kv_heads * d->head_dim * d->elem_bytes;
+    if (strip > 2.0e9L) return false;
+    return true;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool changed = false;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceGuard(int dev)
+    {
+        err = cudaGetDevice(&prev);
+        if (err == cudaSuccess && prev != dev) {
+            err = cudaSetDevice(dev);
+            changed = (err == cudaSuccess);
+        }
+    }
+    ~DeviceGuard()
+    {
+        if (changed) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+struct pdkv_plan {
+    bool has_src = false, has_dst = false;
+    pdkv_pool src{}, dst{};
+    int device = 0;
+    int32_t L = 0, H = 0, D = 0, E = 0, G = 0;
+    int64_t row_bytes = 0, hrow_bytes = 0;
+    int32_t n_req = 0;
+    std::vector<int64_t> kept;      // n_r
+    std::vector<int64_t> req_off;   // bytes, n_req + 1
+    uint64_t payload_bytes = 0, pad_bytes = 0;
+    std::vector<Tile> tiles[3];
+    const Tile *dev_tiles[3] = {nullptr, nullptr, nullptr};
+    std::vector<BlockGroup> groups;
+    void *dev_mem = nullptr;
+    unsigned long long *dev_status = nullptr;
+    int vec_bytes = 16;
+    int sm_count = 1;
+    int lc_fastest = 1;
+};
+
+namespace {
+
+int64_t pool_tile_off(const pdkv_pool_desc &d, int64_t b, int64_t tt, int64_t row, int64_t hrow)
+{
+    if (d.layout == PDKV_LAYOUT_BLOCK_MAJOR)
+        return b * (2 * (int64_t)d.num_layers * d.block_tokens * hrow) + tt * hrow;
+    return b * ((int64_t)d.num_kv_heads * d.block_tokens * row) + tt * row;
+}
+
+pdkv::Side pool_side(const pdkv_pool &p, int64_t row, int64_t hrow)
+{
+    pdkv::Side s;
+    s.base = p.base;
+    s.size = (int64_t)pdkv_pool_bytes(&p.d);
+    if (p.d.layout == PDKV_LAYOUT_BLOCK_MAJOR) {
+        s.lc_stride = (int64_t)p.d.block_tokens * hrow;
+        s.tok_stride = hrow;
+        s.head_stride = row;
+    } else {
+        s.lc_stride = p.d.num_blocks * (int64_t)p.d.num_kv_heads * p.d.block_tokens * row;
+        s.tok_stride = row;
+        s.head_stride = (int64_t)p.d.block_tokens * row;
+    }
+    return s;
+}
+
+pdkv::Side buffer_side(const void *buf, size_t bytes, int64_t row, int64_t hrow)
+{
+    pdkv::Side s;
+    s.base = (char *)buf;
+    s.size = (int64_t)bytes;
+    s.lc_stride = -1;
+    s.tok_stride = hrow;
+    s.head_stride = row;
+    return s;
+}
+
+// Cut the batch into tiles for one operation.  A tile never crosses a block
+// boundary of a paged side it touches, a skip-granule boundary, or the tile
+// size cap; so a tile is all-copy or all-zero, never mixed.
+void build_tiles(pdkv_plan &pl, int op, const pdkv_batch_desc &b, int64_t cap_tok)
+{
+    const bool use_src = op != PDKV_OP_UNPACK, use_dst = op != PDKV_OP_PACK;
+    const int64_t Bp = use_src ? pl.src.d.block_tokens : 0;
+    const int64_t Bd = use_dst ? pl.dst.d.block_tokens : 0;
+    const int64_t G = pl.G;
+    std::vector<Tile> &out = pl.tiles[op];
+    const bool want_groups = op == PDKV_OP_TRANSFER;
+    const bool same_blocks = want_groups && pl.src.d.layout == PDKV_LAYOUT_BLOCK_MAJOR &&
+                             pl.dst.d.layout == PDKV_LAYOUT_BLOCK_MAJOR && Bp == Bd;
+    for (int32_t r = 0; r < pl.n_req; ++r) {
+        const int64_t len = b.seq_len[r];
+        const uint8_t *skip = b.dst_skip ? b.dst_skip + b.dst_tbl_off[r] : nullptr;
+        int64_t t = 0, rank = 0;
+        int64_t group_block = -1;
+        while (t < len) {
+            if (skip && skip[t / G]) {
+                t = std::min(len, (t / G + 1) * G);
+                continue;
+            }
+            int64_t end = std::min(len, t + cap_tok);
+            if (skip) end = std::min(end, (t / G + 1) * G);
+            if (use_src) end = std::min(end, (t / Bp + 1) * Bp);
+            if (use_dst) end = std::min(end, (t / Bd + 1) * Bd);
+            Tile tl;
+            tl.ntok = (int32_t)(end - t);
+            tl.n_kept = (int32_t)pl.kept[r];
+            const int64_t in_buf = pl.req_off[r] + rank * pl.hrow_bytes;
+            tl.src_off = use_src ? pool_tile_off(pl.src.d, b.src_tbl[b.src_tbl_off[r] + t / Bp], t % Bp,
+                                                 pl.row_bytes, pl.hrow_bytes)
+                                 : in_buf;
+            tl.dst_off = use_dst ? pool_tile_off(pl.dst.d, b.dst_tbl[b.dst_tbl_off[r] + t / Bd], t % Bd,
+                                                 pl.row_bytes, pl.hrow_bytes)
+                                 : in_buf;
+            if (want_groups) {
+                if (t / Bp != group_block) {
+                    group_block = t / Bp;
+                    BlockGroup g{};
+                    g.tile_begin = (int32_t)out.size();
+                    g.tile_end = g.tile_begin;
+                    const bool full = same_blocks && (group_block + 1) * Bp <= len;
+                    if (full) {
+                        const int64_t blk = 2 * (int64_t)pl.L * Bp * pl.hrow_bytes;
+                        g.memcpy_src = (int64_t)b.src_tbl[b.src_tbl_off[r] + group_block] * blk;
+                        g.memcpy_dst = (int64_t)b.dst_tbl[b.dst_tbl_off[r] + group_block] * blk;
+                        g.memcpy_bytes = blk;
+                    }
+                    pl.groups.push_back(g);
+                }
+                pl.groups.back().tile_end = (int32_t)out.size() + 1;
+            }
+            out.push_back(tl);
+            rank += end - t;
+            t = end;
+        }
+        if (use_dst && len > 0) {
+            const int64_t nb = (len + Bd - 1) / Bd;
+            const int64_t first_pad = len - (nb - 1) * Bd;
+            if (first_pad < Bd && !(skip && skip[nb - 1])) {
+                const int64_t blk = b.dst_tbl[b.dst_tbl_off[r] + nb - 1];
+                for (int64_t tt = first_pad; tt < Bd; tt += cap_tok) {
+                    Tile tl;
+                    tl.ntok = (int32_t)std::min(cap_tok, Bd - tt);
+                    tl.n_kept = (int32_t)pl.kept[r];
+                    tl.src_off = -1;
+                    tl.dst_off = pool_tile_off(pl.dst.d, blk, tt, pl.row_bytes, pl.hrow_bytes);
+                    out.push_back(tl);
+                    if (want_groups) pl.groups.back().tile_end = (int32_t)out.size();
+                }
+            }
+        }
+    }
+}
+
+int check_table(const int64_t *off, const int32_t *tbl, int32_t n_req, const int32_t *len,
+                int64_t B, int64_t NB)
+{
+    if (!off || !tbl) return PDKV_ERR_INVALID_ARG;
+    if (off[0] < 0) return PDKV_ERR_TABLE;
+    for (int32_t r = 0; r < n_req; ++r) {
+        if (off[r + 1] < off[r]) return PDKV_ERR_TABLE;
+        const int64_t need = ((int64_t)len[r] + B - 1) / B;
+        if (off[r + 1] - off[r] < need) return PDKV_ERR_TABLE;
+        for (int64_t j = 0; j < need; ++j) {
+            const int64_t id = tbl[off[r] + j];
+            if (id < 0 || id >= NB) return PDKV_ERR_TABLE;
+        }
+    }
+    return PDKV_OK;
+}
+
+int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Side &dst,
+              int32_t tile_begin, int32_t n_tiles, int l0, int l1, cudaStream_t stream)
+{
+    if (!pl->dev_mem) return PDKV_ERR_INVALID_ARG;  // host-only plan
+    pdkv::CopyParams p;
+    p.src = src;
+    p.dst = dst;
+    p.tiles = pl->dev_tiles[op];
+    p.tile_begin = tile_begin;
+    p.n_tiles = n_tiles;
+    p.lc_begin = 2 * l0;
+    p.n_lc = 2 * (l1 - l0);
+    p.H = pl->H;
+    p.row_bytes = (int32_t)pl->row_bytes;
+    p.lc_fastest = (int32_t)pdkv::tunables().lc_fastest;
+    p.status = pl->dev_status;
+    pdkv::LaunchConfig cfg;
+    cfg.vec_bytes = pl->vec_bytes;
+    cfg.threads = (int)pdkv::tunables().threads;
+    cfg.ctas_per_sm = (int)pdkv::tunables().ctas_per_sm;
+    cfg.sm_count = pl->sm_count;
+    cfg.variant = (int)pdkv::tunables().variant;
+    cfg.check_bounds = pdkv::tunables().debug_bounds != 0;
+    cudaError_t e = pdkv::launch_copy(p, cfg, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
+    return PDKV_OK;
+}
+
+bool layers_ok(const pdkv_plan *pl, int l0, int l1) { return l0 >= 0 && l0 <= l1 && l1 <= pl->L; }
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+namespace pdkv {
+Tunables &tunables()
+{
+    static Tunables t;
+    return t;
+}
+}  // namespace pdkv
+
+extern "C" {
+
+size_t pdkv_pool_bytes(const pdkv_pool_desc *d)
+{
+    if (!desc_ok(d)) return 0;
+    return (size_t)d->num_blocks * d->num_layers * 2 * d->block_tokens * d->num_kv_heads *
+           d->head_dim * d->elem_bytes;
+}
+
+int pdkv_pool_create(const pdkv_pool_desc *desc, void *dev_base, size_t bytes, int device,
+                     pdkv_pool **out)
+{
+    if (out) *out = nullptr;
+    if (!desc || !out || !dev_base || device < 0) return PDKV_ERR_INVALID_ARG;
+    if (!desc_ok(desc)) return PDKV_ERR_GEOMETRY;
+    if (!aligned16(dev_base) || bytes < pdkv_pool_bytes(desc)) return PDKV_ERR_INVALID_ARG;
+    pdkv_pool *p = new (std::nothrow) pdkv_pool;
+    if (!p) return PDKV_ERR_NOMEM;
+    p->d = *desc;
+    p->base = static_cast<char *>(dev_base);
+    p->bytes = bytes;
+    p->device = device;
+    *out = p;
+    return PDKV_OK;
+}
+
+int pdkv_pool_destroy(pdkv_pool *pool)
+{
+    delete pool;
+    return PDKV_OK;
+}
+
+int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip_granule_tokens,
+                     const pdkv_batch_desc *batch, void *stream, pdkv_plan **out)
+{
+    if (out) *out = nullptr;
+    if (!out || !batch || (!src && !dst)) return PDKV_ERR_INVALID_ARG;
+    if (batch->n_req < 0 || (batch->n_req > 0 && !batch->seq_len)) return PDKV_ERR_INVALID_ARG;
+    if (src && dst) {
+        if (src->d.num_layers != dst->d.num_layers || src->d.num_kv_heads != dst->d.num_kv_heads ||
+            src->d.head_dim != dst->d.head_dim || src->d.elem_bytes != dst->d.elem_bytes)
+            return PDKV_ERR_GEOMETRY;
+        if (src->device != dst->device) return PDKV_ERR_INVALID_ARG;
+    }
+    int32_t G = skip_granule_tokens;
+    if (dst) {
+        if (G <= 0) G = dst->d.block_tokens;
+        if (G != dst->d.block_tokens) return PDKV_ERR_INVALID_ARG;
+    } else if (batch->dst_skip && G <= 0) {
+        return PDKV_ERR_INVALID_ARG;
+    }
+    if (G <= 0) G = 1;
+    for (int32_t r = 0; r < batch->n_req; ++r)
+        if (batch->seq_len[r] < 0) return PDKV_ERR_INVALID_ARG;
+
+    const pdkv_pool *any = src ? src : dst;
+    try {
+        pdkv_plan *pl = new pdkv_plan;
+        struct Holder {
+            pdkv_plan *p;
+            ~Holder() { if (p) pdkv_plan_destroy(p); }
+        } hold{pl};
+        pl->has_src = src != nullptr;
+        pl->has_dst = dst != nullptr;
+        if (src) pl->src = *src;
+        if (dst) pl->dst = *dst;
+        pl->device = any->device;
+        pl->L = any->d.num_layers;
+        pl->H = any->d.num_kv_heads;
+        pl->D = any->d.head_dim;
+        pl->E = any->d.elem_bytes;
+        pl->G = G;
+        pl->row_bytes = (int64_t)pl->D * pl->E;
+        pl->hrow_bytes = pl->row_bytes * pl->H;
+        pl->n_req = batch->n_req;
+        pl->lc_fastest = (int)pdkv::tunables().lc_fastest;
+
+        int rc;
+        if (src && (rc = check_table(batch->src_tbl_off, batch->src_tbl, batch->n_req, batch->seq_len,
+                                     src->d.block_tokens, src->d.num_blocks)) != PDKV_OK)
+            return rc;
+        if (dst && (rc = check_table(batch->dst_tbl_off, batch->dst_tbl, batch->n_req, batch->seq_len,
+                                     dst->d.block_tokens, dst->d.num_blocks)) != PDKV_OK)
+            return rc;
+        if (batch->dst_skip) {
+            if (!batch->dst_tbl_off) return PDKV_ERR_INVALID_ARG;
+            if (batch->dst_tbl_off[0] < 0) return PDKV_ERR_TABLE;
+            for (int32_t r = 0; r < batch->n_req; ++r) {
+                const int64_t need = ((int64_t)batch->seq_len[r] + G - 1) / G;
+                if (batch->dst_tbl_off[r + 1] - batch->dst_tbl_off[r] < need) return PDKV_ERR_TABLE;
+            }
+        }
+        if (dst) {  // every written decode block has exactly one writer
+            std::vector<uint8_t> seen((size_t)dst->d.num_blocks, 0);
+            const int64_t Bd = dst->d.block_tokens;
+            for (int32_t r = 0; r < batch->n_req; ++r) {
+                const int64_t need = ((int64_t)batch->seq_len[r] + Bd - 1) / Bd;
+                for (int64_t j = 0; j < need; ++j) {
+                    const int64_t e = batch->dst_tbl_off[r] + j;
+                    if (batch->dst_skip && batch->dst_skip[e]) continue;
+                    uint8_t &s = seen[(size_t)batch->dst_tbl[e]];
+                    if (s) return PDKV_ERR_TABLE;
+                    s = 1;
+                }
+            }
+        }
+
+        // kept tokens and buffer offsets
+        pl->kept.resize((size_t)pl->n_req);
+        pl->req_off.assign((size_t)pl->n_req + 1, 0);
+        const int64_t tok_bytes = 2 * (int64_t)pl->L * pl->hrow_bytes;
+        uint64_t pad_tokens = 0;
+        for (int32_t r = 0; r < pl->n_req; ++r) {
+            const int64_t len = batch->seq_len[r];
+            int64_t n = len;
+            if (batch->dst_skip) {
+                n = 0;
+                const uint8_t *skip = batch->dst_skip + batch->dst_tbl_off[r];
+                for (int64_t j = 0; j * G < len; ++j)
+                    if (!skip[j]) n += std::min<int64_t>(G, len - j * G);
+            }
+            pl->kept[(size_t)r] = n;
+            pl->req_off[(size_t)r + 1] = pl->req_off[(size_t)r] + n * tok_bytes;
+            if (dst && len > 0) {
+                const int64_t Bd = dst->d.block_tokens;
+                const int64_t nb = (len + Bd - 1) / Bd;
+                if (!(batch->dst_skip && batch->dst_skip[batch->dst_tbl_off[r] + nb - 1]))
+                    pad_tokens += (uint64_t)(nb * Bd - len);
+            }
+        }
+        pl->payload_bytes = (uint64_t)pl->req_off[(size_t)pl->n_req];
+        pl->pad_bytes = pad_tokens * (uint64_t)tok_bytes;
+
+        // widest vector that divides a row (bases are 16-byte aligned)
+        pl->vec_bytes = 16;
+        while (pl->row_bytes % pl->vec_bytes) pl->vec_bytes >>= 1;
+
+        const int64_t cap_tok = std::max<int64_t>(1, pdkv::tunables().tile_bytes / pl->hrow_bytes);
+        if (src) build_tiles(*pl, PDKV_OP_PACK, *batch, cap_tok);
+        if (dst) build_tiles(*pl, PDKV_OP_UNPACK, *batch, cap_tok);
+        if (src && dst) build_tiles(*pl, PDKV_OP_TRANSFER, *batch, cap_tok);
+        for (int op = 0; op < 3; ++op)
+            if (pl->tiles[op].size() > (size_t)INT32_MAX) return PDKV_ERR_INVALID_ARG;
+
+        if (pdkv::tunables().dry_run) {  // host-only plan: tile lists can be inspected, nothing can launch
+            hold.p = nullptr;
+            *out = pl;
+            return PDKV_OK;
+        }
+
+        // one device allocation: [status words][pack tiles][unpack tiles][transfer tiles]
+        DeviceGuard guard(pl->device);
+        if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+        cudaDeviceProp prop;
+        cudaError_t e = cudaGetDeviceProperties(&prop, pl->device);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetDeviceProperties");
+        pl->sm_count = prop.multiProcessorCount;
+        const size_t head = 256;
+        size_t total = head;
+        for (int op = 0; op < 3; ++op) total += pl->tiles[op].size() * sizeof(Tile);
+        e = cudaMalloc(&pl->dev_mem, total);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc");
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        e = cudaMemsetAsync(pl->dev_mem, 0, head, st);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+        pl->dev_status = static_cast<unsigned long long *>(pl->dev_mem);
+        size_t at = head;
+        for (int op = 0; op < 3; ++op) {
+            const size_t bytes = pl->tiles[op].size() * sizeof(Tile);
+            pl->dev_tiles[op] = reinterpret_cast<const Tile *>(static_cast<char *>(pl->dev_mem) + at);
+            if (bytes) {
+                e = cudaMemcpyAsync(static_cast<char *>(pl->dev_mem) + at, pl->tiles[op].data(), bytes,
+                                    cudaMemcpyHostToDevice, st);
+                if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync");
+            }
+            at += bytes;
+        }
+        e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+        hold.p = nullptr;
+        *out = pl;
+        return PDKV_OK;
+    } catch (const std::bad_alloc &) {
+        return PDKV_ERR_NOMEM;
+    }
+}
+
+int pdkv_plan_destroy(pdkv_plan *plan)
+{
+    if (!plan) return PDKV_OK;
+    int rc = PDKV_OK;
+    if (plan->dev_mem) {
+        DeviceGuard guard(plan->device);
+        cudaError_t e = cudaFree(plan->dev_mem);
+        if (e != cudaSuccess) rc = cuda_fail(e, "cudaFree");
+    }
+    delete plan;
+    return rc;
+}
+
+int pdkv_plan_buffer(const pdkv_plan *plan, size_t *total_bytes, const int64_t **req_off_bytes)
+{
+    if (!plan) return PDKV_ERR_INVALID_ARG;
+    if (total_bytes) *total_bytes = (size_t)plan->payload_bytes;
+    if (req_off_bytes) *req_off_bytes = plan->req_off.data();
+    return PDKV_OK;
+}
+
+int pdkv_plan_traffic(const pdkv_plan *plan, int op, uint64_t *bytes_read, uint64_t *bytes_written)
+{
+    if (!plan || op < 0 || op > 2) return PDKV_ERR_INVALID_ARG;
+    if ((op != PDKV_OP_UNPACK && !plan->has_src) || (op != PDKV_OP_PACK && !plan->has_dst))
+        return PDKV_ERR_INVALID_ARG;
+    if (bytes_read) *bytes_read = plan->payload_bytes;
+    if (bytes_written) *bytes_written = plan->payload_bytes + (op == PDKV_OP_PACK ? 0 : plan->pad_bytes);
+    return PDKV_OK;
+}
+
+int pdkv_pack(const pdkv_plan *plan, void *buf, size_t buf_bytes, int l0, int l1, void *stream)
+{
+    if (!plan || !plan->has_src || !layers_ok(plan, l0, l1)) return PDKV_ERR_INVALID_ARG;
+    if (buf_bytes < plan->payload_bytes) return PDKV_ERR_BUFFER_TOO_SMALL;
+    if (!plan->dev_mem) return PDKV_ERR_INVALID_ARG;  // host-only plan
+    if (plan->payload_bytes == 0 || l0 == l1) return PDKV_OK;
+    if (!buf || !aligned16(buf)) return PDKV_ERR_INVALID_ARG;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    return launch_op(plan, PDKV_OP_PACK, pool_side(plan->src, plan->row_bytes, plan->hrow_bytes),
+                     buffer_side(buf, buf_bytes, plan->row_bytes, plan->hrow_bytes), 0,
+                     (int32_t)plan->tiles[PDKV_OP_PACK].size(), l0, l1, static_cast<cudaStream_t>(stream));
+}
+
+int pdkv_unpack(const pdkv_plan *plan, const void *buf, size_t buf_bytes, int l0, int l1, void *stream)
+{
+    if (!plan || !plan->has_dst || !layers_ok(plan, l0, l1)) return PDKV_ERR_INVALID_ARG;
+    if (buf_bytes < plan->payload_bytes) return PDKV_ERR_BUFFER_TOO_SMALL;
+    if (!plan->dev_mem) return PDKV_ERR_INVALID_ARG;  // host-only plan
+    if (plan->tiles[PDKV_OP_UNPACK].empty() || l0 == l1) return PDKV_OK;
+    if (plan->payload_bytes && (!buf || !aligned16(buf))) return PDKV_ERR_INVALID_ARG;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    return launch_op(plan, PDKV_OP_UNPACK, buffer_side(buf, buf_bytes, plan->row_bytes, plan->hrow_bytes),
+                     pool_side(plan->dst, plan->row_bytes, plan->hrow_bytes), 0,
+                     (int32_t)plan->tiles[PDKV_OP_UNPACK].size(), l0, l1,
+                     static_cast<cudaStream_t>(stream));
+}
+
+int pdkv_transfer(const pdkv_plan *plan, int l0, int l1, void *stream)
+{
+    if (!plan || !plan->has_src || !plan->has_dst || !layers_ok(plan, l0, l1))
+        return PDKV_ERR_INVALID_ARG;
+    if (!plan->dev_mem) return PDKV_ERR_INVALID_ARG;  // host-only plan
+    if (plan->tiles[PDKV_OP_TRANSFER].empty() || l0 == l1) return PDKV_OK;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    return launch_op(plan, PDKV_OP_TRANSFER, pool_side(plan->src, plan->row_bytes, plan->hrow_bytes),
+                     pool_side(plan->dst, plan->row_bytes, plan->hrow_bytes), 0,
+                     (int32_t)plan->tiles[PDKV_OP_TRANSFER].size(), l0, l1,
+                     static_cast<cudaStream_t>(stream));
+}
+
+int pdkv_transfer_blockwise(const pdkv_plan *plan, void *stream)
+{
+    if (!plan || !plan->has_src || !plan->has_dst || !plan->dev_mem) return PDKV_ERR_INVALID_ARG;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const pdkv::Side s = pool_side(plan->src, plan->row_bytes, plan->hrow_bytes);
+    const pdkv::Side d = pool_side(plan->dst, plan->row_bytes, plan->hrow_bytes);
+    for (const BlockGroup &g : plan->groups) {
+        if (g.memcpy_bytes > 0) {
+            cudaError_t e = cudaMemcpyAsync(plan->dst.base + g.memcpy_dst, plan->src.base + g.memcpy_src,
+                                            (size_t)g.memcpy_bytes, cudaMemcpyDeviceToDevice, st);
+            if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync");
+        } else {
+            int rc = launch_op(plan, PDKV_OP_TRANSFER, s, d, g.tile_begin, g.tile_end - g.tile_begin, 0,
+                               plan->L, st);
+            if (rc != PDKV_OK) return rc;
+        }
+    }
+    return PDKV_OK;
+}
+
+int pdkv_plan_launches(const pdkv_plan *plan, int op, int64_t *launches)
+{
+    if (!plan || !launches || op < 0 || op > 3) return PDKV_ERR_INVALID_ARG;
+    if (op == 3)
+        *launches = (int64_t)plan->groups.size();
+    else
+        *launches = plan->tiles[op].empty() ? 0 : 1;
+    return PDKV_OK;
+}
+
+int pdkv_plan_tiles(const pdkv_plan *plan, int op, const pdkv_tile **tiles, int64_t *n_tiles)
+{
+    if (!plan || op < 0 || op > 2 || !tiles || !n_tiles) return PDKV_ERR_INVALID_ARG;
+    static_assert(sizeof(pdkv_tile) == sizeof(Tile), "public and internal tile records must match");
+    *tiles = reinterpret_cast<const pdkv_tile *>(plan->tiles[op].data());
+    *n_tiles = (int64_t)plan->tiles[op].size();
+    return PDKV_OK;
+}
+
+int pdkv_plan_status(const pdkv_plan *plan, void *stream)
+{
+    if (!plan || !plan->dev_mem) return PDKV_ERR_INVALID_ARG;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    unsigned long long word[2] = {0, 0};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(word, plan->dev_status, sizeof(word), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e, "status read");
+    if (word[0]) {
+        char msg[96];
+        std::snprintf(msg, sizeof(msg), "refused access at byte offset %lld", (long long)word[1]);
+        g_cuda_msg = msg;
+        return PDKV_ERR_DEVICE_BOUNDS;
+    }
+    return PDKV_OK;
+}
+
+int pdkv_tune(const char *key, int64_t value)
+{
+    if (!key) return PDKV_ERR_INVALID_ARG;
+    pdkv::Tunables &t = pdkv::tunables();
+    const std::string k(key);
+    if (k == "tile_bytes" && value >= 1 && value <= (1ll << 30)) t.tile_bytes = value;
+    else if (k == "ctas_per_sm" && value >= 1 && value <= 32) t.ctas_per_sm = value;
+    else if (k == "threads" && value >= 32 && value <= 1024 && value % 32 == 0) t.threads = value;
+    else if (k == "lc_fastest" && (value == 0 || value == 1)) t.lc_fastest = value;
+    else if (k == "debug_bounds" && (value == 0 || value == 1)) t.debug_bounds = value;
+    else if (k == "variant" && value >= 0 && value <= 1) t.variant = value;
+    else if (k == "dry_run" && (value == 0 || value == 1)) t.dry_run = value;
+    else return PDKV_ERR_INVALID_ARG;
+    return PDKV_OK;
+}
+
+int pdkv_tune_get(const char *key, int64_t *value)
+{
+    if (!key || !value) return PDKV_ERR_INVALID_ARG;
+    const pdkv::Tunables &t = pdkv::tunables();
+    const std::string k(key);
+    if (k == "tile_bytes") *value = t.tile_bytes;
+    else if (k == "ctas_per_sm") *value = t.ctas_per_sm;
+    else if (k == "threads") *value = t.threads;
+    else if (k == "lc_fastest") *value = t.lc_fastest;
+    else if (k == "debug_bounds") *value = t.debug_bounds;
+    else if (k == "variant") *value = t.variant;
+    else if (k == "dry_run") *value = t.dry_run;
+    else return PDKV_ERR_INVALID_ARG;
+    return PDKV_OK;
+}
+
+const char *pdkv_strerror(int status)
+{
+    switch (status) {
+    case PDKV_OK: return "ok";
+    case PDKV_ERR_INVALID_ARG: return "invalid argument";
+    case PDKV_ERR_GEOMETRY: return "invalid or mismatched pool geometry";
+    case PDKV_ERR_TABLE: return "invalid block table";
+    case PDKV_ERR_BUFFER_TOO_SMALL: return "contiguous buffer too small";
+    case PDKV_ERR_CUDA: return g_cuda_msg.empty() ? "CUDA error" : g_cuda_msg.c_str();
+    case PDKV_ERR_DEVICE_BOUNDS: return g_cuda_msg.empty() ? "device bounds check refused an access" : g_cuda_msg.c_str();
+    case PDKV_ERR_NOMEM: return "out of host memory";
+    default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,67 @@
+// Internal declarations shared by the host planner and the kernel launchers.
+#pragma once
+
+#include <cstdint>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "pdkv.h"
+
+namespace pdkv {
+
+// One unit of work along the token axis: `ntok` consecutive kept tokens of one
+// request that lie inside one block on every paged side of the copy.  Offsets
+// are bytes from the side's base for layer 0 / K; the kernel adds the (l, c)
+// step.  src_off < 0 marks a zero-fill tile (tail slots of a last decode block).
+struct Tile {
+    int64_t src_off;
+    int64_t dst_off;
+    int32_t ntok;
+    int32_t n_kept;  // kept tokens of the request: the buffer's per-(l,c) stride is n_kept * H * ROW
+};
+
+// Addressing of one side of a copy (a pool in either layout, or the buffer).
+struct Side {
+    char *base;
+    int64_t size;         // addressable bytes, for the bounds-checked build of the kernels
+    int64_t lc_stride;    // bytes per (l,c) step; < 0: request dependent (contiguous buffer)
+    int64_t tok_stride;   // bytes between consecutive tokens of one head
+    int64_t head_stride;  // bytes between consecutive heads of one token
+};
+
+struct CopyParams {
+    Side src, dst;
+    const Tile *tiles;
+    int32_t tile_begin, n_tiles;
+    int32_t lc_begin, n_lc;
+    int32_t H;
+    int32_t row_bytes;   // D * E
+    int32_t lc_fastest;
+    unsigned long long *status;  // [0] != 0: an access was refused; [1] offending offset
+};
+
+struct LaunchConfig {
+    int vec_bytes;   // 16, 8, 4, 2 or 1
+    int threads;
+    int ctas_per_sm;
+    int sm_count;
+    int variant;
+    bool check_bounds;
+};
+
+// Enqueue one persistent copy kernel.  Returns the CUDA status of the launch.
+cudaError_t launch_copy(const CopyParams &p, const LaunchConfig &cfg, cudaStream_t stream);
+
+struct Tunables {
+    int64_t tile_bytes = 65536;
+    int64_t ctas_per_sm = 4;
+    int64_t threads = 512;
+    int64_t lc_fastest = 1;
+    int64_t debug_bounds = 0;
+    int64_t variant = 0;
+    int64_t dry_run = 0;
+};
+Tunables &tunables();
+
+}  // namespace pdkv

@@ -1,0 +1,208 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU checker,
+bit for bit, on the same seeded inputs.  Sizes here finish in seconds on the
+checker yet span many tiles, ragged tails, both layouts, skip masks, layer
+ranges and the narrow-vector fallbacks."""
+import numpy as np
+import pytest
+
+from paper_2408_08147_b200 import binding as B
+from paper_2408_08147_b200 import workloads as W
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+SENT = W.SENTINEL_U16
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _gpu_lib():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    B.lib()                      # must exist: no fallback
+    B.pdkv_tune("dry_run", 0)
+    B.pdkv_tune("debug_bounds", 0)
+    yield
+    B.pdkv_tune("debug_bounds", 0)
+    B.pdkv_tune("tile_bytes", 65536)
+    B.pdkv_tune("lc_fastest", 1)
+
+
+def dev(a: np.ndarray):
+    return torch.from_numpy(a.reshape(-1).view(np.uint8).copy()).cuda()
+
+
+def host(t, dtype=np.uint16):
+    return t.cpu().numpy().view(dtype)
+
+
+def check_all_ops(oracle, w, *, layers=None, elem_dtype=np.uint16, side_stream=False,
+                  blockwise=True, bounds=False):
+    """Run pack, unpack, fused and block-by-block on the GPU and compare every
+    byte (owned and untouched) with the checker."""
+    from paper_2408_08147_b200.session import TransferSession
+
+    G = w.dst.block_tokens
+    src = W.fill_pool_numpy(w.src, w.seed)
+    sent = W.sentinel_pool_numpy(w.dst)
+    n_buf = oracle.buffer_elems(w.batch, G, w.src)
+    slack = 64
+
+    want_buf = np.full(n_buf + slack, sent[0], elem_dtype)
+    oracle.pack(w.src, src, w.batch, G, want_buf, layers=layers)
+    full_buf = np.zeros(n_buf + slack, elem_dtype)
+    oracle.pack(w.src, src, w.batch, G, full_buf)
+    want_dst = sent.copy()
+    oracle.unpack(w.dst, want_dst, w.batch, full_buf, layers=layers)
+
+    B.pdkv_tune("debug_bounds", 1 if bounds else 0)
+    stream = torch.cuda.Stream() if side_stream else torch.cuda.current_stream()
+    src_t, dst_t = dev(src), dev(sent)
+    buf_t = dev(np.full(n_buf + slack, sent[0], elem_dtype))
+    torch.cuda.synchronize()
+    with TransferSession(w.src, src_t, w.dst, dst_t, w.batch, stream.cuda_stream) as s:
+        assert s.buffer_bytes == n_buf * w.src.elem_bytes
+        s.pack(buf_t, layers)
+        s.status()
+        assert np.array_equal(host(buf_t, elem_dtype), want_buf), "pack"
+        assert np.array_equal(host(src_t, elem_dtype), src), "pack wrote the source pool"
+
+        fb_t = dev(full_buf)
+        s.unpack(fb_t, layers)
+        s.status()
+        assert np.array_equal(host(dst_t, elem_dtype), want_dst), "unpack"
+
+        dst_t.copy_(dev(sent))
+        s.transfer(layers)
+        s.status()
+        assert np.array_equal(host(dst_t, elem_dtype), want_dst), "fused transfer"
+
+        if blockwise and layers is None:
+            dst_t.copy_(dev(sent))
+            s.transfer_blockwise()
+            s.status()
+            assert np.array_equal(host(dst_t, elem_dtype), want_dst), "block-by-block baseline"
+    B.pdkv_tune("debug_bounds", 0)
+
+
+def test_config1_tiny_bounds_checked_then_plain(oracle):
+    w = W.make_config(1)
+    check_all_ops(oracle, w, bounds=True)
+    check_all_ops(oracle, w, bounds=False, side_stream=True)
+    check_all_ops(oracle, w, layers=(1, 2))
+
+
+@pytest.mark.parametrize("idx,kw", [
+    (2, dict(num_layers=2, n_req=5, max_len=640)),                       # A->A, equal blocks
+    (2, dict(num_layers=2, n_req=5, max_len=600, src_layout=W.LAYER_MAJOR)),  # B->B
+    (3, dict(num_layers=2, n_req=12, max_len=1500)),                     # 16 -> 128 re-blocking
+    (4, dict(num_layers=3, n_req=4, max_len=700)),                       # fragmented pool, 64 -> 128
+    (5, dict(num_layers=2, n_req=40)),                                   # skip mask
+    (5, dict(num_layers=2, n_req=24, src_block=256)),                    # prefill block > decode block
+    (3, dict(num_layers=2, n_req=6, max_len=900, src_layout=W.LAYER_MAJOR,
+             dst_layout=W.BLOCK_MAJOR)),                                 # B -> A
+])
+def test_scaled_configs(oracle, idx, kw):
+    w = W.make_config(idx, **kw)
+    check_all_ops(oracle, w, bounds=True)
+    check_all_ops(oracle, w)
+
+
+@pytest.mark.parametrize("tile_bytes,lc_fastest", [(2048, 1), (16384, 0), (1 << 20, 1)])
+def test_tile_size_and_work_order_do_not_change_the_result(oracle, tile_bytes, lc_fastest):
+    B.pdkv_tune("tile_bytes", tile_bytes)
+    B.pdkv_tune("lc_fastest", lc_fastest)
+    try:
+        check_all_ops(oracle, W.make_config(3, num_layers=2, n_req=8, max_len=1200))
+        check_all_ops(oracle, W.make_config(5, num_layers=1, n_req=30, src_block=32))
+    finally:
+        B.pdkv_tune("tile_bytes", 65536)
+        B.pdkv_tune("lc_fastest", 1)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_small_geometries(oracle, seed):
+    """Odd block sizes, non-power-of-two heads, rows narrower than 16 bytes,
+    1-, 4- and 8-byte elements, random skip masks, zero-length requests."""
+    rng = np.random.default_rng(9000 + seed)
+    E = int(rng.choice([1, 2, 2, 4, 8]))
+    D = int(rng.choice([1, 2, 4, 8, 24, 64]))
+    lens = rng.integers(0, 90, size=int(rng.integers(1, 7))).astype(np.int32)
+    w = W.build_workload("rnd", int(rng.integers(1 << 30)), num_layers=int(rng.integers(1, 4)),
+                         num_kv_heads=int(rng.integers(1, 6)), head_dim=D, elem_bytes=E,
+                         seq_len=lens, src_layout=int(rng.integers(2)),
+                         src_block=int(rng.choice([1, 3, 7, 16, 48])),
+                         dst_layout=int(rng.integers(2)),
+                         dst_block=int(rng.choice([2, 5, 16, 32, 64])),
+                         src_slack=1.4, dst_slack=1.4)
+    if seed % 2 and w.batch.dst_tbl.size:
+        w.batch.dst_skip = (rng.random(w.batch.dst_tbl.size) < 0.3).astype(np.uint8)
+    dt = {1: np.uint8, 2: np.uint16, 4: np.uint32, 8: np.uint64}[E]
+    L = w.src.num_layers
+    layers = None if seed % 3 else (L - 1, L)
+    check_all_ops(oracle, w, elem_dtype=dt, layers=layers, bounds=True)
+    check_all_ops(oracle, w, elem_dtype=dt, layers=layers)
+
+
+def test_empty_and_degenerate_batches(oracle):
+    from paper_2408_08147_b200.session import TransferSession
+
+    g_src = W.Geometry(W.BLOCK_MAJOR, 2, 2, 16, 2, 4, 6)
+    g_dst = W.Geometry(W.LAYER_MAJOR, 2, 2, 16, 2, 8, 4)
+    sent_t = dev(W.sentinel_pool_numpy(g_dst))
+    src_t = dev(W.fill_pool_numpy(g_src, 1))
+    z64, z32 = np.zeros(1, np.int64), np.zeros(0, np.int32)
+    # no requests at all
+    empty = W.Batch(z32, z64, z32, z64, z32)
+    dst_t = sent_t.clone()
+    with TransferSession(g_src, src_t, g_dst, dst_t, empty) as s:
+        assert s.buffer_bytes == 0
+        buf_t = torch.zeros(16, dtype=torch.uint8, device="cuda")
+        s.pack(buf_t); s.unpack(buf_t); s.transfer(); s.transfer_blockwise(); s.status()
+        assert s.launches(B.PDKV_OP_TRANSFER) == 0
+    assert torch.equal(dst_t, sent_t)
+    # zero-length requests and a request whose blocks are all resident
+    lens = np.array([0, 8, 0], np.int32)
+    bt = W.Batch(lens, np.array([0, 0, 2, 2], np.int64), np.array([1, 4], np.int32),
+                 np.array([0, 0, 1, 1], np.int64), np.array([2], np.int32),
+                 np.array([1], np.uint8))
+    with TransferSession(g_src, src_t, g_dst, dst_t, bt) as s:
+        assert s.buffer_bytes == 0
+        s.transfer(); s.transfer_blockwise(); s.status()
+    assert torch.equal(dst_t, sent_t)
+    # a whole-model call with an empty layer range does nothing
+    bt.dst_skip = None
+    with TransferSession(g_src, src_t, g_dst, dst_t, bt) as s:
+        s.transfer((1, 1)); s.status()
+        assert torch.equal(dst_t, sent_t)
+        s.transfer()
+        want = W.sentinel_pool_numpy(g_dst)
+        oracle.transfer(g_src, host(src_t), g_dst, want, bt)
+        assert np.array_equal(host(dst_t), want)
+
+
+def test_per_layer_calls_equal_whole_model(oracle):
+    """Sec. 3.5: per-layer or whole-model transfer differ only in offset and
+    length; issuing the layers one by one must give the same bytes."""
+    from paper_2408_08147_b200.session import TransferSession
+
+    w = W.make_config(3, num_layers=4, n_req=5, max_len=500)
+    src = W.fill_pool_numpy(w.src, w.seed)
+    sent = W.sentinel_pool_numpy(w.dst)
+    want = sent.copy()
+    oracle.transfer(w.src, src, w.dst, want, w.batch)
+    src_t, dst_t = dev(src), dev(sent)
+    with TransferSession(w.src, src_t, w.dst, dst_t, w.batch) as s:
+        buf_t = torch.zeros(s.buffer_bytes, dtype=torch.uint8, device="cuda")
+        streams = [torch.cuda.Stream() for _ in range(2)]
+        torch.cuda.synchronize()
+        for l in range(4):                      # layers alternate between two streams
+            st = streams[l % 2]
+            s.pack(buf_t, (l, l + 1), st.cuda_stream)
+            s.unpack(buf_t, (l, l + 1), st.cuda_stream)
+        torch.cuda.synchronize()
+        assert np.array_equal(host(dst_t), want)
+        dst_t.copy_(dev(sent))
+        for l in reversed(range(4)):
+            s.transfer((l, l + 1))
+        s.status()
+        assert np.array_equal(host(dst_t), want)

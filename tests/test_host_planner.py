@@ -1,0 +1,267 @@
+"""Host-side logic of the library, no GPU needed: exported symbols, argument
+validation, buffer offsets, traffic accounting, and the tile lists (executed by
+a small numpy interpreter and compared with the CPU checker)."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2408_08147_b200 import binding as B
+from paper_2408_08147_b200 import build as pdkv_build
+from paper_2408_08147_b200 import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SENT = W.SENTINEL_U16
+FAKE_BASE = 0x7F0000000000  # never dereferenced: dry-run plans make no CUDA call
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    pdkv_build.build_library()
+    B.pdkv_tune("dry_run", 1)
+    yield
+    B.pdkv_tune("dry_run", 0)
+    B.pdkv_tune("tile_bytes", 65536)
+
+
+def test_library_exports_every_declared_symbol():
+    with open(os.path.join(ROOT, "include", "pdkv.h")) as f:
+        text = f.read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(pdkv_[a-z_]+)\s*\(", text))
+    assert {"pdkv_pool_create", "pdkv_pack", "pdkv_unpack", "pdkv_transfer"} <= declared
+    lib = B.lib()
+    for name in declared:
+        assert hasattr(lib, name), f"{name} declared in pdkv.h but not exported"
+    assert declared == set(B.EXPORTS)
+
+
+def _pools(w):
+    ps = B.pdkv_pool_create(B.desc_of(w.src), FAKE_BASE, w.src.num_bytes(), 0)
+    pd = B.pdkv_pool_create(B.desc_of(w.dst), FAKE_BASE + (1 << 40), w.dst.num_bytes(), 0)
+    return ps, pd
+
+
+def _plan(w, ps, pd, **over):
+    b = w.batch
+    kw = dict(seq_len=b.seq_len, src_tbl_off=b.src_tbl_off, src_tbl=b.src_tbl,
+              dst_tbl_off=b.dst_tbl_off, dst_tbl=b.dst_tbl, dst_skip=b.dst_skip)
+    kw.update(over)
+    return B.pdkv_plan_create(ps, pd, w.dst.block_tokens, **kw)
+
+
+def test_pool_validation():
+    good = B.make_desc(0, 2, 4, 64, 2, 16, 10)
+    assert B.pdkv_pool_bytes(good) == 10 * 2 * 2 * 16 * 4 * 64 * 2
+    for bad in [B.make_desc(2, 2, 4, 64, 2, 16, 10), B.make_desc(0, 0, 4, 64, 2, 16, 10),
+                B.make_desc(0, 2, 4, 64, 3, 16, 10), B.make_desc(0, 2, 4, 64, 2, 0, 10),
+                B.make_desc(0, 2, 4, 64, 2, 16, 0), B.make_desc(0, 2, -1, 64, 2, 16, 10)]:
+        assert B.pdkv_pool_bytes(bad) == 0
+        with pytest.raises(B.PdkvError) as e:
+            B.pdkv_pool_create(bad, FAKE_BASE, 1 << 30, 0)
+        assert e.value.status == B.PDKV_ERR_GEOMETRY
+    with pytest.raises(B.PdkvError) as e:
+        B.pdkv_pool_create(good, FAKE_BASE + 8, 1 << 30, 0)       # misaligned
+    assert e.value.status == B.PDKV_ERR_INVALID_ARG
+    with pytest.raises(B.PdkvError) as e:
+        B.pdkv_pool_create(good, FAKE_BASE, B.pdkv_pool_bytes(good) - 1, 0)  # too small
+    assert e.value.status == B.PDKV_ERR_INVALID_ARG
+    with pytest.raises(B.PdkvError) as e:
+        B.pdkv_pool_create(good, 0, 1 << 30, 0)
+    assert e.value.status == B.PDKV_ERR_INVALID_ARG
+
+
+def test_plan_validation_errors():
+    w = W.make_config(1)
+    ps, pd = _pools(w)
+    b = w.batch
+
+    def status(**over):
+        with pytest.raises(B.PdkvError) as e:
+            _plan(w, ps, pd, **over)
+        return e.value.status
+
+    t = b.src_tbl.copy(); t[3] = w.src.num_blocks
+    assert status(src_tbl=t) == B.PDKV_ERR_TABLE
+    t = b.src_tbl.copy(); t[0] = -1
+    assert status(src_tbl=t) == B.PDKV_ERR_TABLE
+    t = b.dst_tbl.copy(); t[1] = t[0]
+    assert status(dst_tbl=t) == B.PDKV_ERR_TABLE                   # two writers for one block
+    off = b.src_tbl_off.copy(); off[1:] -= 1
+    off[1] = max(off[1], 0)
+    assert status(src_tbl_off=off) == B.PDKV_ERR_TABLE             # a table is too short
+    off = b.dst_tbl_off.copy(); off[2] = off[1] - 1
+    assert status(dst_tbl_off=off) == B.PDKV_ERR_TABLE             # not monotone
+    ln = b.seq_len.copy(); ln[0] = -5
+    assert status(seq_len=ln) == B.PDKV_ERR_INVALID_ARG
+    assert status(src_tbl=None) == B.PDKV_ERR_INVALID_ARG
+    # duplicate prefill blocks are legal (shared prefix on the sender)
+    t = b.src_tbl.copy(); t[1] = t[0]
+    B.pdkv_plan_destroy(_plan(w, ps, pd, src_tbl=t))
+    # geometry mismatch between the two pools
+    other = B.pdkv_pool_create(B.make_desc(1, 3, 4, 64, 2, 32, w.dst.num_blocks), FAKE_BASE,
+                               1 << 40, 0)
+    with pytest.raises(B.PdkvError) as e:
+        _plan(w, ps, other)
+    assert e.value.status == B.PDKV_ERR_GEOMETRY
+    # skip granule must be the decode block
+    with pytest.raises(B.PdkvError) as e:
+        B.pdkv_plan_create(ps, pd, 16, b.seq_len, b.src_tbl_off, b.src_tbl, b.dst_tbl_off, b.dst_tbl)
+    assert e.value.status == B.PDKV_ERR_INVALID_ARG
+    with pytest.raises(B.PdkvError) as e:
+        B.pdkv_plan_create(None, None, 0, b.seq_len)
+    assert e.value.status == B.PDKV_ERR_INVALID_ARG
+    for p in (ps, pd, other):
+        B.pdkv_pool_destroy(p)
+
+
+def test_launch_argument_errors_and_dry_run_refusal():
+    w = W.make_config(1)
+    ps, pd = _pools(w)
+    plan = _plan(w, ps, pd)
+    total, _ = B.pdkv_plan_buffer(plan)
+    for fn, args in [(B.pdkv_pack, (plan, FAKE_BASE, total, 0, 3)),
+                     (B.pdkv_pack, (plan, FAKE_BASE, total, -1, 1)),
+                     (B.pdkv_unpack, (plan, FAKE_BASE, total, 2, 1)),
+                     (B.pdkv_pack, (plan, FAKE_BASE + 4, total, 0, 2)),
+                     (B.pdkv_transfer, (plan, 0, 5))]:
+        with pytest.raises(B.PdkvError) as e:
+            fn(*args)
+        assert e.value.status == B.PDKV_ERR_INVALID_ARG
+    with pytest.raises(B.PdkvError) as e:
+        B.pdkv_pack(plan, FAKE_BASE, total - 1, 0, 2)
+    assert e.value.status == B.PDKV_ERR_BUFFER_TOO_SMALL
+    # a dry-run plan owns no device arrays: launching is refused, not attempted
+    for fn, args in [(B.pdkv_pack, (plan, FAKE_BASE, total, 0, 2)),
+                     (B.pdkv_transfer, (plan, 0, 2)), (B.pdkv_transfer_blockwise, (plan,)),
+                     (B.pdkv_plan_status, (plan,))]:
+        with pytest.raises(B.PdkvError) as e:
+            fn(*args)
+        assert e.value.status == B.PDKV_ERR_INVALID_ARG
+    # pack-only plans cannot unpack
+    ponly = B.pdkv_plan_create(ps, None, 32, w.batch.seq_len, w.batch.src_tbl_off, w.batch.src_tbl)
+    with pytest.raises(B.PdkvError) as e:
+        B.pdkv_unpack(ponly, FAKE_BASE, total, 0, 2)
+    assert e.value.status == B.PDKV_ERR_INVALID_ARG
+    assert B.pdkv_plan_buffer(ponly)[0] == total
+    for p in (plan, ponly):
+        B.pdkv_plan_destroy(p)
+    B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
+    assert "table" in B.pdkv_strerror(B.PDKV_ERR_TABLE)
+    with pytest.raises(B.PdkvError):
+        B.pdkv_tune("no_such_key", 1)
+    with pytest.raises(B.PdkvError):
+        B.pdkv_tune("threads", 33)
+
+
+# --------------------------------------------------------------------------
+# tile lists, executed in numpy
+# --------------------------------------------------------------------------
+
+def _side(geom):
+    row = geom.head_dim * geom.elem_bytes
+    hrow = row * geom.num_kv_heads
+    if geom.layout == W.BLOCK_MAJOR:
+        return geom.block_tokens * hrow, hrow, row
+    return geom.num_blocks * geom.num_kv_heads * geom.block_tokens * row, row, geom.block_tokens * row
+
+
+def run_tiles(tiles, src_bytes, src_side, dst_bytes, dst_side, geom, layers):
+    """Apply a tile list the way the header documents it; also proves that no
+    destination byte is written twice."""
+    row = geom.head_dim * geom.elem_bytes
+    hrow = row * geom.num_kv_heads
+    written = np.zeros(dst_bytes.shape[0], bool)
+    for t in tiles:
+        for lc in range(2 * layers[0], 2 * layers[1]):
+            s_lc, s_tok, s_head = src_side if src_side else (t["n_kept"] * hrow, hrow, row)
+            d_lc, d_tok, d_head = dst_side if dst_side else (t["n_kept"] * hrow, hrow, row)
+            for tk in range(t["ntok"]):
+                for h in range(geom.num_kv_heads):
+                    d = t["dst_off"] + lc * d_lc + tk * d_tok + h * d_head
+                    assert not written[d:d + row].any()
+                    written[d:d + row] = True
+                    if t["src_off"] < 0:
+                        dst_bytes[d:d + row] = 0
+                    else:
+                        s = t["src_off"] + lc * s_lc + tk * s_tok + h * s_head
+                        dst_bytes[d:d + row] = src_bytes[s:s + row]
+    return written
+
+
+def _random_workload(rng, skip):
+    L = int(rng.integers(1, 3)); H = int(rng.integers(1, 4)); D = int(rng.choice([4, 8, 16]))
+    lens = rng.integers(0, 40, size=int(rng.integers(1, 5))).astype(np.int32)
+    w = W.build_workload("t", int(rng.integers(1 << 30)), num_layers=L, num_kv_heads=H,
+                         head_dim=D, elem_bytes=2, seq_len=lens,
+                         src_layout=int(rng.integers(2)), src_block=int(rng.choice([1, 3, 4, 8, 16])),
+                         dst_layout=int(rng.integers(2)), dst_block=int(rng.choice([2, 4, 5, 8, 32])),
+                         src_slack=1.3, dst_slack=1.3)
+    if skip and w.batch.dst_tbl.size:
+        w.batch.dst_skip = (rng.random(w.batch.dst_tbl.size) < 0.35).astype(np.uint8)
+    return w
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_tile_lists_reproduce_the_checker(oracle, seed):
+    rng = np.random.default_rng(4242 + seed)
+    w = _random_workload(rng, skip=bool(seed % 2))
+    B.pdkv_tune("tile_bytes", int(rng.choice([64, 256, 4096, 65536])))
+    ps, pd = _pools(w)
+    plan = _plan(w, ps, pd)
+    G = w.dst.block_tokens
+    g = w.src
+    layers = (0, g.num_layers) if seed % 3 else (g.num_layers - 1, g.num_layers)
+
+    src = W.fill_pool_numpy(w.src, w.seed)
+    n_buf = oracle.buffer_elems(w.batch, G, w.src)
+    total, offs = B.pdkv_plan_buffer(plan, w.batch.n_req)
+    assert total == n_buf * 2
+    assert np.array_equal(offs, oracle.request_offsets(w.batch, G, w.src) * 2)
+
+    want_buf = np.full(n_buf, SENT, np.uint16)
+    oracle.pack(w.src, src, w.batch, G, want_buf, layers=layers)
+    got_buf = np.full(n_buf, SENT, np.uint16)
+    run_tiles(B.pdkv_plan_tiles(plan, B.PDKV_OP_PACK), src.view(np.uint8), _side(w.src),
+              got_buf.view(np.uint8), None, g, layers)
+    assert np.array_equal(got_buf, want_buf)
+
+    full_buf = np.zeros(n_buf, np.uint16)
+    oracle.pack(w.src, src, w.batch, G, full_buf)
+    want_dst = W.sentinel_pool_numpy(w.dst)
+    oracle.unpack(w.dst, want_dst, w.batch, full_buf, layers=layers)
+    got_dst = W.sentinel_pool_numpy(w.dst)
+    run_tiles(B.pdkv_plan_tiles(plan, B.PDKV_OP_UNPACK), full_buf.view(np.uint8), None,
+              got_dst.view(np.uint8), _side(w.dst), g, layers)
+    assert np.array_equal(got_dst, want_dst)
+
+    got_dst = W.sentinel_pool_numpy(w.dst)
+    written = run_tiles(B.pdkv_plan_tiles(plan, B.PDKV_OP_TRANSFER), src.view(np.uint8),
+                        _side(w.src), got_dst.view(np.uint8), _side(w.dst), g, layers)
+    assert np.array_equal(got_dst, want_dst)
+
+    if layers == (0, g.num_layers):
+        rd, wr = B.pdkv_plan_traffic(plan, B.PDKV_OP_TRANSFER)
+        assert rd == total and wr == int(written.sum())
+        assert B.pdkv_plan_traffic(plan, B.PDKV_OP_PACK) == (total, total)
+    B.pdkv_plan_destroy(plan)
+    B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
+
+
+def test_tiles_respect_size_cap_and_block_boundaries():
+    w = W.make_config(3, num_layers=2, n_req=6, max_len=700)
+    B.pdkv_tune("tile_bytes", 16384)
+    ps, pd = _pools(w)
+    plan = _plan(w, ps, pd)
+    hrow = w.src.num_kv_heads * w.src.head_dim * w.src.elem_bytes
+    for op in (B.PDKV_OP_PACK, B.PDKV_OP_UNPACK, B.PDKV_OP_TRANSFER):
+        tiles = B.pdkv_plan_tiles(plan, op)
+        assert tiles["ntok"].min() >= 1 and tiles["ntok"].max() * hrow <= 16384
+        copy = tiles[tiles["src_off"] >= 0]
+        assert copy["ntok"].sum() == w.batch.seq_len.sum()
+    n_blocks = int((-(-w.batch.seq_len.astype(np.int64) // 16)).sum())
+    assert B.pdkv_plan_launches(plan, B.PDKV_OP_BLOCKWISE) == n_blocks
+    assert B.pdkv_plan_launches(plan, B.PDKV_OP_TRANSFER) == 1
+    B.pdkv_plan_destroy(plan)
+    B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
