@@ -1,0 +1,533 @@
+#!/usr/bin/env python
+"""Benchmark of the paged-KVCache transfer path.
+
+One *step* is one pass of the whole hot path over one batch: pack (blocks ->
+contiguous buffer), unpack (buffer -> decode blocks) and the fused
+blocks-to-blocks transfer, each one library call.  The reported value is the
+algorithmic traffic of a step (payload read + payload written + zero padding
+written, summed over the three calls) divided by the device time of the step.
+
+    python bench.py --gpus 1 --steps 50 --warmup 5            # this library
+    python bench.py --impl reference --steps 3 --warmup 1      # CPU checker arm
+
+Prints exactly one JSON line on stdout (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "KV pack+unpack+fused transfer throughput (algorithmic bytes read+written)"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+KERNEL_SOURCE = os.path.join(ROOT, "paper_2408_08147_b200", "csrc", "pdkv_kernels.cu")
+
+# DRAM traffic per launch from ncu (dram__bytes_read.sum + dram__bytes_write.sum),
+# keyed by (workload, op); valid only while the kernel source hashes to KERNEL_SHA.
+NCU_TRAFFIC: dict = {}
+NCU_KERNEL_SHA = ""
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def kernel_sha() -> str:
+    with open(KERNEL_SOURCE, "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:16]
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while a region runs
+    (read-only queries; nothing is set)."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception as e:  # pragma: no cover
+            log(f"[bench] NVML unavailable: {e}")
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thr:
+            self._thr.join()
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------------
+# distributed plumbing (one process per GPU; no data-path collective)
+# ---------------------------------------------------------------------------
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), \
+        int(os.environ.get("WORLD_SIZE", 1))
+
+
+def dist_init(backend: str):
+    import torch.distributed as dist
+
+    rank, _, world = dist_env()
+    if world > 1 and not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, world
+
+
+def barrier():
+    import torch.distributed as dist
+
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+def reduce_step_time(ms_local: float, units_local: float, device=None):
+    """Max of the per-rank times and sum of the per-rank units, on every rank."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()):
+        return ms_local, units_local
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    u = torch.tensor([units_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# ---------------------------------------------------------------------------
+# workload on the device
+# ---------------------------------------------------------------------------
+
+def workload_name(w):
+    s, d = w.src, w.dst
+    lay = {0: "block-major", 1: "layer-major"}
+    return (f"{w.name}: L={s.num_layers} H={s.num_kv_heads} D={s.head_dim} E={s.elem_bytes} "
+            f"{w.batch.n_req} req x {int(w.batch.seq_len.sum())} tokens; prefill {lay[s.layout]} "
+            f"B={s.block_tokens} NB={s.num_blocks}; decode {lay[d.layout]} B={d.block_tokens} "
+            f"NB={d.num_blocks}")
+
+
+def alloc_pools(w, torch, seed_offset=0):
+    from paper_2408_08147_b200 import workloads as W
+
+    src_t = torch.empty(w.src.num_bytes(), dtype=torch.uint8, device="cuda")
+    W.fill_pool_torch(src_t, w.seed + seed_offset)
+    dst_t = torch.empty(w.dst.num_bytes(), dtype=torch.uint8, device="cuda")
+    dst_t.view(torch.int16).fill_(W.SENTINEL_U16 - 65536 if W.SENTINEL_U16 > 32767 else W.SENTINEL_U16)
+    return src_t, dst_t
+
+
+def token_major_torch(geom, pool_t, tbl, length, torch):
+    """[L][2][len][H][D] view-copy of one request, through reshape/index/permute
+    (an independent cross-check of the kernels; not the CPU checker)."""
+    v = pool_t.view(torch.int16).view(geom.shape())
+    B = geom.block_tokens
+    nb = -(-length // B)
+    idx = torch.as_tensor(tbl[:nb].astype("int64"), device=pool_t.device)
+    if geom.layout == 0:
+        x = v[idx].permute(1, 2, 0, 3, 4, 5)
+    else:
+        x = v[:, :, idx].permute(0, 1, 2, 4, 3, 5)
+    L, H, D = geom.num_layers, geom.num_kv_heads, geom.head_dim
+    return x.reshape(L, 2, nb * B, H, D)[:, :, :length]
+
+
+def sanity_check(w, src_t, dst_t, torch) -> bool:
+    """A few requests' tokens must be identical in both pools after a transfer."""
+    b = w.batch
+    if b.dst_skip is not None:
+        return True
+    for r in sorted({0, b.n_req // 2, b.n_req - 1}):
+        n = int(b.seq_len[r])
+        s = token_major_torch(w.src, src_t, b.src_tbl[b.src_tbl_off[r]:b.src_tbl_off[r + 1]], n, torch)
+        d = token_major_torch(w.dst, dst_t, b.dst_tbl[b.dst_tbl_off[r]:b.dst_tbl_off[r + 1]], n, torch)
+        if not torch.equal(s, d):
+            return False
+    return True
+
+
+# ---------------------------------------------------------------------------
+# CPU checker legs
+# ---------------------------------------------------------------------------
+
+def oracle_step(O, sub, src_np, dst_np, buf_np, threads):
+    G = sub.dst.block_tokens
+    O.pack(sub.src, src_np, sub.batch, G, buf_np, threads=threads)
+    O.unpack(sub.dst, dst_np, sub.batch, buf_np, threads=threads)
+    O.transfer(sub.src, src_np, sub.dst, dst_np, sub.batch, threads=threads)
+
+
+def step_bytes_of(w):
+    """Algorithmic bytes of one step, from the batch alone (no skip: payload and padding)."""
+    import numpy as np
+
+    tok = w.src.token_bytes()
+    b = w.batch
+    lens = b.seq_len.astype(np.int64)
+    Bd = w.dst.block_tokens
+    nblk = -(-lens // Bd)
+    if b.dst_skip is None:
+        kept = int(lens.sum())
+        pad = int((nblk * Bd - lens).sum())
+    else:
+        kept = pad = 0
+        for r in range(b.n_req):
+            sk = b.dst_skip[b.dst_tbl_off[r]:b.dst_tbl_off[r] + nblk[r]]
+            for j in range(int(nblk[r])):
+                if not sk[j]:
+                    kept += int(min(Bd, lens[r] - j * Bd))
+            if nblk[r] and not sk[nblk[r] - 1]:
+                pad += int(nblk[r] * Bd - lens[r])
+    P = kept * tok
+    return 2 * P + (2 * P + pad * tok) * 2
+
+
+def cpu_baseline(w, src_t, budget_s=20.0):
+    """Time the CPU checker, as it stands, on the first requests of the batch."""
+    import numpy as np
+
+    from oracle import pdkv_oracle as O
+    from paper_2408_08147_b200 import workloads as W
+
+    cores = os.cpu_count() or 1
+    n = min(w.batch.n_req, cores, 8)
+    # keep the sample near `budget_s` CPU-seconds at ~0.4 GB/s per thread
+    tok_bytes = w.src.token_bytes()
+    while n > 1 and 6 * int(w.batch.seq_len[:n].sum()) * tok_bytes / 0.4e9 > 2 * budget_s:
+        n -= 1
+    sub, s_ids, _ = W.compact_subproblem(w, range(n))
+    src_np = W.gather_blocks(src_t.view(__import__("torch").int16), w.src, s_ids).cpu().numpy().view(np.uint16)
+    dst_np = W.sentinel_pool_numpy(sub.dst)
+    buf_np = np.zeros(O.buffer_elems(sub.batch, sub.dst.block_tokens, sub.src), np.uint16)
+    threads = min(cores, n)
+    t0 = time.perf_counter()
+    oracle_step(O, sub, src_np, dst_np, buf_np, threads)
+    dt = time.perf_counter() - t0
+    nbytes = step_bytes_of(sub)
+    return {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"first {n} of {w.batch.n_req} requests ({int(sub.batch.seq_len.sum())} tokens, "
+                      f"all layers), one pack+unpack+fused pass, {dt:.2f} s wall",
+            "host_cpus": cores}
+
+
+def reference_arm(args):
+    """The CPU checker timed as the reference implementation (rank 0 only)."""
+    import numpy as np
+
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    from oracle import pdkv_oracle as O
+    from paper_2408_08147_b200 import workloads as W
+
+    cores = os.cpu_count() or 1
+    full = W.make_config(args.config)
+    # bounded sample: whole run (warmup + steps) within ~2 minutes at ~0.4 GB/s per thread
+    per_step_s = max(0.5, 110.0 / (args.steps + args.warmup))
+    threads = min(cores, 8, full.batch.n_req)
+    tok = full.src.token_bytes()
+    tokens_budget = per_step_s * threads * 0.4e9 / (6 * tok)
+    n_req = max(1, min(threads, full.batch.n_req))
+    layers = full.src.num_layers
+    while layers > 1 and float(full.batch.seq_len[:n_req].sum()) * layers / full.src.num_layers > tokens_budget:
+        layers = max(1, layers // 2)
+    w = W.make_config(args.config, n_req=n_req, num_layers=layers)
+    chunk = W.normal_bf16_bits(1 << 22, w.seed)
+    src_np = np.resize(chunk, w.src.num_elems())
+    dst_np = W.sentinel_pool_numpy(w.dst)
+    buf_np = np.zeros(O.buffer_elems(w.batch, w.dst.block_tokens, w.src), np.uint16)
+    for _ in range(args.warmup):
+        oracle_step(O, w, src_np, dst_np, buf_np, threads)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(O, w, src_np, dst_np, buf_np, threads)
+    dt = time.perf_counter() - t0
+    nbytes = step_bytes_of(w)
+    value = nbytes * args.steps / dt / 1e9
+    sample = (f"{n_req} of {full.batch.n_req} requests, {layers} of {full.src.num_layers} layers "
+              f"per step ({nbytes / 1e9:.2f} GB algorithmic), {threads} threads")
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+           "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+           "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "u16", "data": "synthetic",
+           "config": {"workload": workload_name(full), "sample": sample},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                            "sample": sample},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+# ---------------------------------------------------------------------------
+# main arm
+# ---------------------------------------------------------------------------
+
+def main_arm(args):
+    import numpy as np
+    import torch
+
+    from paper_2408_08147_b200 import binding as B
+    from paper_2408_08147_b200 import workloads as W
+    from paper_2408_08147_b200.session import TransferSession
+
+    B.lib()  # fail loudly if the CUDA library is missing
+    rank, local, world = dist_env()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    torch.cuda.set_device(local)
+    rank, world = dist_init("nccl")
+    dev = torch.device("cuda", local)
+
+    for k, v in (args.tune or []):
+        B.pdkv_tune(k, int(v))
+
+    kw = {}
+    if args.src_block:
+        kw["src_block"] = args.src_block
+    if args.layouts:
+        kw["src_layout"], kw["dst_layout"] = ("AB".index(args.layouts[0]), "AB".index(args.layouts[1]))
+    w = W.make_config(args.config, **kw)
+    src_t, dst_t = alloc_pools(w, torch, seed_offset=rank)
+    stream = torch.cuda.Stream()
+    sess = TransferSession(w.src, src_t, w.dst, dst_t, w.batch, stream.cuda_stream)
+    buf_t = torch.empty(max(sess.buffer_bytes, 16), dtype=torch.uint8, device=dev)
+    ops = [("pack", B.PDKV_OP_PACK, lambda: sess.pack(buf_t)),
+           ("unpack", B.PDKV_OP_UNPACK, lambda: sess.unpack(buf_t)),
+           ("fused", B.PDKV_OP_TRANSFER, lambda: sess.transfer())]
+    traffic = {name: sum(sess.traffic(op)) for name, op, _ in ops}
+    step_bytes = sum(traffic.values())
+    launches_per_step = sum(sess.launches(op) for _, op, _ in ops)
+
+    def run_step(evs=None):
+        for i, (_, _, fn) in enumerate(ops):
+            if evs is not None:
+                evs[i].record(stream)
+            fn()
+        if evs is not None:
+            evs[3].record(stream)
+
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            run_step()
+    torch.cuda.synchronize()
+    sess.status()
+    ok = sanity_check(w, src_t, dst_t, torch)
+
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local) as clk:
+        with torch.cuda.stream(stream):
+            for k in range(args.steps):
+                run_step(evs[k])
+        torch.cuda.synchronize()
+    barrier()
+    total_ms = evs[0][0].elapsed_time(evs[-1][3])
+    op_ms = {name: statistics.fmean(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps))
+             for i, (name, _, _) in enumerate(ops)}
+    op_best = {name: min(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps))
+               for i, (name, _, _) in enumerate(ops)}
+    ms_step_local = total_ms / args.steps
+    ms_step, units = reduce_step_time(ms_step_local, float(step_bytes), dev)
+    value = units / (ms_step * 1e-3) / 1e9
+
+    peak, peak_kind = measured_peak()
+    per_op = {}
+    for name, _, _ in ops:
+        ach = traffic[name] / (op_ms[name] * 1e-3) / 1e9
+        per_op[name] = {"ms": op_ms[name], "ms_best": op_best[name], "GBps": ach,
+                        "frac_of_" + peak_kind: ach / peak, "frac_of_nominal_8000": ach / 8000.0,
+                        "bytes": traffic[name]}
+    dom = max(per_op, key=lambda n: per_op[n]["ms"])
+    sha = kernel_sha()
+    traffic_ncu = NCU_TRAFFIC.get((args.config, dom)) if sha == NCU_KERNEL_SHA else None
+    roofline = {"bound": "hbm", "achieved": per_op[dom]["GBps"], "peak": peak, "unit": "GB/s",
+                "frac": per_op[dom]["GBps"] / peak, "traffic": traffic_ncu, "op": dom,
+                "kernel": "pdkv::copy_tiles_kernel", "peak_source": f"{peak_kind} (MEASURED_PEAKS.json hbm_gbs)"
+                if peak_kind == "measured" else "fallback 6650 GB/s",
+                "algorithmic_bytes_per_launch": traffic[dom]}
+
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "u16", "data": "synthetic",
+           "config": {"workload": workload_name(w), "config_index": args.config,
+                      "step": "pdkv_pack + pdkv_unpack + pdkv_transfer, all layers",
+                      "payload_bytes": sess.buffer_bytes, "step_bytes": step_bytes,
+                      "l2": "inputs exceed L2 (pools and buffer are GiB-sized; no flush needed)"
+                      if sess.buffer_bytes > (1 << 29) else "L2-resident workload: not an HBM number",
+                      "tunables": {k: B.pdkv_tune_get(k) for k in
+                                   ("tile_bytes", "ctas_per_sm", "threads", "lc_fastest", "variant")}},
+           "ops": per_op, "roofline": roofline, "gpu_launches": launches_per_step * args.steps,
+           "sanity_check": "ok" if ok else "MISMATCH", "clocks": clk.summary()}
+
+    if rank == 0 and not args.no_extras:
+        # block-by-block baseline (Sec. 2.3 "transfer one by one"): same result, host loop
+        n_blk = sess.launches(B.PDKV_OP_BLOCKWISE)
+        reps = max(1, min(5, args.steps))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            sess.transfer_blockwise()
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for _ in range(reps):
+                sess.transfer_blockwise()
+            e1.record(stream)
+        torch.cuda.synchronize()
+        bw_ms = e0.elapsed_time(e1) / reps
+        out["blockwise_baseline"] = {"ms": bw_ms, "GBps": traffic["fused"] / (bw_ms * 1e-3) / 1e9,
+                                     "gpu_ops_per_call": n_blk,
+                                     "fused_speedup": bw_ms / op_ms["fused"]}
+
+    # end to end: pinned host pools, H2D of the prefill pool, plan, the three calls, D2H of the decode pool
+    if not args.no_extras:
+        try:
+            out["e2e"] = e2e_leg(args, w, src_t, dst_t, buf_t, stream, step_bytes, torch, B, TransferSession, dev)
+        except Exception as e:  # pragma: no cover
+            out["e2e"] = {"error": repr(e)}
+    sess.close()
+
+    if rank == 0 and world == 1 and not args.no_extras and not args.no_cpu:
+        try:
+            out["cpu_baseline"] = cpu_baseline(w, src_t)
+        except Exception as e:  # pragma: no cover
+            out["cpu_baseline"] = {"error": repr(e)}
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.destroy_process_group()
+
+
+def e2e_leg(args, w, src_t, dst_t, buf_t, stream, step_bytes, torch, B, TransferSession, dev):
+    """Same step, but the prefill pool starts in pinned host memory and the
+    decode pool is read back to pinned host memory, every step, inside the timed
+    region; the plan (tables) is also rebuilt from host arrays each step."""
+    free_host = None
+    try:
+        import psutil
+
+        free_host = psutil.virtual_memory().available
+    except Exception:
+        pass
+    need = src_t.numel() + dst_t.numel()
+    if free_host is not None and need > 0.6 * free_host:
+        return {"value": None, "unit": UNIT, "skipped": f"needs {need >> 30} GiB pinned host memory"}
+    h_src = torch.empty(src_t.numel(), dtype=torch.uint8, pin_memory=True)
+    h_dst = torch.empty(dst_t.numel(), dtype=torch.uint8, pin_memory=True)
+    h_src.copy_(src_t)
+    steps = max(1, min(args.e2e_steps, args.steps))
+
+    def one():
+        with torch.cuda.stream(stream):
+            src_t.copy_(h_src, non_blocking=True)
+            s = TransferSession(w.src, src_t, w.dst, dst_t, w.batch, stream.cuda_stream)
+            s.pack(buf_t)
+            s.unpack(buf_t)
+            s.transfer()
+            h_dst.copy_(dst_t, non_blocking=True)
+        stream.synchronize()
+        s.close()
+
+    one()
+    barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one()
+    torch.cuda.synchronize()
+    barrier()
+    ms = (time.perf_counter() - t0) * 1e3 / steps
+    ms, units = reduce_step_time(ms, float(step_bytes), dev)
+    del h_src, h_dst
+    return {"value": units / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms, "steps": steps,
+            "h2d_bytes_per_step": int(src_t.numel()), "d2h_bytes_per_step": int(dst_t.numel()),
+            "includes": "H2D prefill pool from pinned memory, pdkv_plan_create, pack, unpack, fused, "
+                        "D2H decode pool to pinned memory"}
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="pdkv", choices=["pdkv", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="workload 1..5 (2 = the headline config)")
+    ap.add_argument("--src-block", type=int, default=0)
+    ap.add_argument("--layouts", default="", help="two letters, e.g. AB: prefill block-major, decode layer-major")
+    ap.add_argument("--tune", nargs=2, action="append", metavar=("KEY", "VALUE"))
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-extras", action="store_true", help="skip baseline, e2e and CPU legs")
+    ap.add_argument("--no-cpu", action="store_true")
+    return ap.parse_args()
+
+
+if __name__ == "__main__":
+    a = parse()
+    a.warmup = max(a.warmup, 3) if a.impl == "pdkv" else a.warmup
+    if a.impl == "reference":
+        reference_arm(a)
+    else:
+        main_arm(a)

@@ -289,3 +289,65 @@ def fill_pool_torch(pool, seed: int) -> None:
     g = torch.Generator(device=pool.device)
     g.manual_seed(seed)
     pool.view(torch.bfloat16).normal_(generator=g)
+
+
+# ---------------------------------------------------------------------------
+# sub-problems: a few requests of a large batch with their blocks renumbered
+# ---------------------------------------------------------------------------
+
+def compact_subproblem(w: Workload, req_ids):
+    """Requests ``req_ids`` of ``w`` as a self-contained workload.
+
+    Block ids are renumbered 0..k-1 in order of first appearance, so the pools
+    of the sub-problem hold just the gathered blocks.  Returns the new workload
+    and the original prefill / decode block ids in compact order; pair it with
+    :func:`gather_blocks` to build the compact pools.  Only bookkeeping happens
+    here (no element of KV is touched).
+    """
+    b = w.batch
+    req_ids = [int(r) for r in req_ids]
+
+    def renumber(off, tbl):
+        ids, new_tbl, counts, seen = [], [], [], {}
+        for r in req_ids:
+            ent = tbl[off[r]:off[r + 1]]
+            counts.append(len(ent))
+            for e in ent:
+                e = int(e)
+                if e not in seen:
+                    seen[e] = len(ids)
+                    ids.append(e)
+                new_tbl.append(seen[e])
+        return (_csr(np.asarray(counts, np.int64)), np.asarray(new_tbl, np.int32),
+                np.asarray(ids, np.int64))
+
+    s_off, s_tbl, s_ids = renumber(b.src_tbl_off, b.src_tbl)
+    d_off, d_tbl, d_ids = renumber(b.dst_tbl_off, b.dst_tbl)
+    skip = None
+    if b.dst_skip is not None:
+        skip = np.concatenate([b.dst_skip[b.dst_tbl_off[r]:b.dst_tbl_off[r + 1]] for r in req_ids]
+                              or [np.zeros(0, np.uint8)]).astype(np.uint8)
+    nb = Batch(b.seq_len[req_ids].astype(np.int32), s_off, s_tbl, d_off, d_tbl, skip)
+    src = replace(w.src, num_blocks=max(1, len(s_ids)))
+    dst = replace(w.dst, num_blocks=max(1, len(d_ids)))
+    return Workload(w.name + "-sub", w.seed, src, dst, nb, note=w.note), s_ids, d_ids
+
+
+def gather_blocks(pool, geom: Geometry, ids):
+    """Blocks ``ids`` of a flat pool (torch tensor or numpy array of raw
+    elements) as a new flat compact pool, through a reshaped view."""
+    n = len(ids)
+    if n == 0:
+        shape = replace(geom, num_blocks=1).shape()
+        return pool[:0].new_zeros(int(np.prod(shape))) if hasattr(pool, "new_zeros") \
+            else np.zeros(int(np.prod(shape)), pool.dtype)
+    v = pool.reshape(geom.shape())
+    if hasattr(pool, "new_zeros"):
+        import torch
+
+        idx = torch.as_tensor(np.asarray(ids, np.int64), device=pool.device)
+        out = v[idx] if geom.layout == BLOCK_MAJOR else v[:, :, idx]
+        return out.contiguous().reshape(-1)
+    idx = np.asarray(ids, np.int64)
+    out = v[idx] if geom.layout == BLOCK_MAJOR else v[:, :, idx]
+    return np.ascontiguousarray(out).reshape(-1)
