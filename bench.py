@@ -346,6 +346,10 @@ def main_arm(args):
     kw = {}
     if args.src_block:
         kw["src_block"] = args.src_block
+    if args.n_req:
+        kw["n_req"] = args.n_req
+    if args.num_layers:
+        kw["num_layers"] = args.num_layers
     if args.layouts:
         kw["src_layout"], kw["dst_layout"] = ("AB".index(args.layouts[0]), "AB".index(args.layouts[1]))
     w = W.make_config(args.config, **kw)
@@ -418,7 +422,7 @@ def main_arm(args):
                       "l2": "inputs exceed L2 (pools and buffer are GiB-sized; no flush needed)"
                       if sess.buffer_bytes > (1 << 29) else "L2-resident workload: not an HBM number",
                       "tunables": {k: B.pdkv_tune_get(k) for k in
-                                   ("tile_bytes", "ctas_per_sm", "threads", "lc_fastest", "variant")}},
+                                   ("tile_bytes", "ctas_per_sm", "threads", "unroll", "vec32", "lc_fastest", "variant")}},
            "ops": per_op, "roofline": roofline, "gpu_launches": launches_per_step * args.steps,
            "sanity_check": "ok" if ok else "MISMATCH", "clocks": clk.summary()}
 
@@ -516,6 +520,8 @@ def parse():
     ap.add_argument("--impl", default="pdkv", choices=["pdkv", "reference"])
     ap.add_argument("--config", type=int, default=2, help="workload 1..5 (2 = the headline config)")
     ap.add_argument("--src-block", type=int, default=0)
+    ap.add_argument("--n-req", type=int, default=0, help="shrink the batch (profiling captures)")
+    ap.add_argument("--num-layers", type=int, default=0, help="shrink the model (profiling captures)")
     ap.add_argument("--layouts", default="", help="two letters, e.g. AB: prefill block-major, decode layer-major")
     ap.add_argument("--tune", nargs=2, action="append", metavar=("KEY", "VALUE"))
     ap.add_argument("--e2e-steps", type=int, default=3)

@@ -196,9 +196,13 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream);
 
 /* Process-wide tunables, read when a plan is created or a call is launched:
  *   "tile_bytes"     target bytes moved per tile (default 65536)
- *   "ctas_per_sm"    persistent CTAs per SM (default 4)
- *   "threads"        threads per CTA, multiple of 32 (default 512)
- *   "lc_fastest"     1: consecutive work items walk layers of one tile (default 1)
+ *   "ctas_per_sm"    persistent CTAs per SM (default 2)
+ *   "threads"        threads per CTA, multiple of 32 (default 512; clamped to
+ *                    what the register budget of the chosen variant allows)
+ *   "unroll"         independent accesses in flight per thread: 1, 2, 4, 8 (default 1)
+ *   "vec32"          1: use 32-byte accesses when rows and bases allow (default 1)
+ *   "lc_fastest"     1: consecutive work items walk the (layer, K/V) strips of
+ *                    one tile; 0: they walk the tiles of one strip (default 0)
  *   "debug_bounds"   1: kernels range-check every access and skip bad ones
  *   "variant"        0: register copy, 1: bulk async copy through shared memory
  *   "dry_run"        1: pdkv_plan_create builds host-only plans (no CUDA call is

@@ -243,6 +243,10 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     p.status = pl->dev_status;
     pdkv::LaunchConfig cfg;
     cfg.vec_bytes = pl->vec_bytes;
+    if (pl->vec_bytes == 16 && pdkv::tunables().vec32 && pl->row_bytes % 32 == 0 &&
+        ((reinterpret_cast<uintptr_t>(src.base) | reinterpret_cast<uintptr_t>(dst.base)) & 31u) == 0)
+        cfg.vec_bytes = 32;
+    cfg.unroll = (int)pdkv::tunables().unroll;
     cfg.threads = (int)pdkv::tunables().threads;
     cfg.ctas_per_sm = (int)pdkv::tunables().ctas_per_sm;
     cfg.sm_count = pl->sm_count;
@@ -404,7 +408,21 @@ int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip_gr
         pl->vec_bytes = 16;
         while (pl->row_bytes % pl->vec_bytes) pl->vec_bytes >>= 1;
 
-        const int64_t cap_tok = std::max<int64_t>(1, pdkv::tunables().tile_bytes / pl->hrow_bytes);
+        // Tile size cap.  The kernels split a vector index with multiply-high
+        // divisions that are exact while dividend * divisor < 2^32, so the cap
+        // also keeps vectors * vectors-per-row and rows * max(H, tokens) below it.
+        int64_t cap_tok = std::max<int64_t>(1, pdkv::tunables().tile_bytes / pl->hrow_bytes);
+        {
+            const int64_t vpr = pl->row_bytes / pl->vec_bytes;
+            const int64_t max_b = std::max<int64_t>(src ? src->d.block_tokens : 1, dst ? dst->d.block_tokens : 1);
+            auto exact = [&](int64_t cap) {
+                const long double tok = (long double)std::min(cap, max_b);
+                const long double rows = tok * pl->H;
+                return rows * vpr * vpr < 4.0e9L && rows * std::max<long double>(pl->H, tok) < 4.0e9L;
+            };
+            while (cap_tok > 1 && !exact(cap_tok)) cap_tok /= 2;
+            if (!exact(cap_tok)) return PDKV_ERR_GEOMETRY;
+        }
         if (src) build_tiles(*pl, PDKV_OP_PACK, *batch, cap_tok);
         if (dst) build_tiles(*pl, PDKV_OP_UNPACK, *batch, cap_tok);
         if (src && dst) build_tiles(*pl, PDKV_OP_TRANSFER, *batch, cap_tok);
@@ -596,6 +614,8 @@ int pdkv_tune(const char *key, int64_t value)
     if (k == "tile_bytes" && value >= 1 && value <= (1ll << 30)) t.tile_bytes = value;
     else if (k == "ctas_per_sm" && value >= 1 && value <= 32) t.ctas_per_sm = value;
     else if (k == "threads" && value >= 32 && value <= 1024 && value % 32 == 0) t.threads = value;
+    else if (k == "unroll" && (value == 1 || value == 2 || value == 4 || value == 8)) t.unroll = value;
+    else if (k == "vec32" && (value == 0 || value == 1)) t.vec32 = value;
     else if (k == "lc_fastest" && (value == 0 || value == 1)) t.lc_fastest = value;
     else if (k == "debug_bounds" && (value == 0 || value == 1)) t.debug_bounds = value;
     else if (k == "variant" && value >= 0 && value <= 1) t.variant = value;
@@ -612,6 +632,8 @@ int pdkv_tune_get(const char *key, int64_t *value)
     if (k == "tile_bytes") *value = t.tile_bytes;
     else if (k == "ctas_per_sm") *value = t.ctas_per_sm;
     else if (k == "threads") *value = t.threads;
+    else if (k == "unroll") *value = t.unroll;
+    else if (k == "vec32") *value = t.vec32;
     else if (k == "lc_fastest") *value = t.lc_fastest;
     else if (k == "debug_bounds") *value = t.debug_bounds;
     else if (k == "variant") *value = t.variant;

@@ -42,7 +42,8 @@ struct CopyParams {
 };
 
 struct LaunchConfig {
-    int vec_bytes;   // 16, 8, 4, 2 or 1
+    int vec_bytes;   // 32, 16, 8, 4, 2 or 1
+    int unroll;      // independent accesses per thread: 1, 2, 4 or 8
     int threads;
     int ctas_per_sm;
     int sm_count;
@@ -55,9 +56,11 @@ cudaError_t launch_copy(const CopyParams &p, const LaunchConfig &cfg, cudaStream
 
 struct Tunables {
     int64_t tile_bytes = 65536;
-    int64_t ctas_per_sm = 4;
+    int64_t ctas_per_sm = 2;
     int64_t threads = 512;
-    int64_t lc_fastest = 1;
+    int64_t unroll = 1;
+    int64_t vec32 = 1;
+    int64_t lc_fastest = 0;
     int64_t debug_bounds = 0;
     int64_t variant = 0;
     int64_t dry_run = 0;

@@ -4,13 +4,20 @@
 //
 // The path is pure data movement (Sec. 3.5: organise blocks into a contiguous
 // buffer, restore blocks from bytes), so the only resource that matters is HBM
-// bandwidth: accesses are 16 bytes per lane, every warp touches whole rows, and
-// each thread keeps several independent loads in flight before storing.
+// bandwidth: accesses are 32 (or 16) bytes per lane, every warp touches whole
+// rows, and the number of bytes each SM keeps in flight is a launch parameter
+// (threads x CTAs x unroll), because on B200 a copy runs fastest with about
+// 32-64 KiB of loads outstanding per SM, not with as many as fit.
 #include "pdkv_internal.h"
 
 namespace pdkv {
 
+struct alignas(32) Vec32 {
+    unsigned int a[8];
+};
+
 template <int W> struct VecT;
+template <> struct VecT<32> { using type = Vec32; };
 template <> struct VecT<16> { using type = uint4; };
 template <> struct VecT<8> { using type = uint2; };
 template <> struct VecT<4> { using type = unsigned int; };
@@ -18,14 +25,48 @@ template <> struct VecT<2> { using type = unsigned short; };
 template <> struct VecT<1> { using type = unsigned char; };
 
 template <typename V> __device__ __forceinline__ V zero_vec();
+template <> __device__ __forceinline__ Vec32 zero_vec<Vec32>()
+{
+    Vec32 v;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v.a[i] = 0u;
+    return v;
+}
 template <> __device__ __forceinline__ uint4 zero_vec<uint4>() { return make_uint4(0, 0, 0, 0); }
 template <> __device__ __forceinline__ uint2 zero_vec<uint2>() { return make_uint2(0, 0); }
 template <> __device__ __forceinline__ unsigned int zero_vec<unsigned int>() { return 0u; }
 template <> __device__ __forceinline__ unsigned short zero_vec<unsigned short>() { return 0; }
 template <> __device__ __forceinline__ unsigned char zero_vec<unsigned char>() { return 0; }
 
-constexpr int kMaxThreads = 512;
-constexpr int kUnroll = 8;
+// Threads per CTA the register budget allows: W*U/4 data registers per thread
+// plus addressing must stay below 65536 / threads.
+constexpr int max_threads(int w, int u) { return w * u >= 256 ? 256 : (w * u >= 128 ? 512 : 1024); }
+
+// Streaming (evict-first) global accesses; the 32-byte forms are single
+// 256-bit instructions on sm_100.
+template <typename V> __device__ __forceinline__ V ld_stream(const char *p)
+{
+    return __ldcs(reinterpret_cast<const V *>(p));
+}
+template <> __device__ __forceinline__ Vec32 ld_stream<Vec32>(const char *p)
+{
+    Vec32 v;
+    asm volatile("ld.global.cs.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(v.a[0]), "=r"(v.a[1]), "=r"(v.a[2]), "=r"(v.a[3]), "=r"(v.a[4]), "=r"(v.a[5]),
+                   "=r"(v.a[6]), "=r"(v.a[7])
+                 : "l"(p));
+    return v;
+}
+template <typename V> __device__ __forceinline__ void st_stream(char *p, const V &v)
+{
+    __stcs(reinterpret_cast<V *>(p), v);
+}
+template <> __device__ __forceinline__ void st_stream<Vec32>(char *p, const Vec32 &v)
+{
+    asm volatile("st.global.cs.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};" ::"r"(v.a[0]), "r"(v.a[1]),
+                 "r"(v.a[2]), "r"(v.a[3]), "r"(v.a[4]), "r"(v.a[5]), "r"(v.a[6]), "r"(v.a[7]), "l"(p)
+                 : "memory");
+}
 
 __device__ __forceinline__ bool in_bounds(int64_t off, int width, int64_t size)
 {
@@ -37,13 +78,24 @@ __device__ __forceinline__ void refuse(unsigned long long *status, int64_t off)
     if (atomicCAS(status, 0ull, 1ull) == 0ull) status[1] = (unsigned long long)off;
 }
 
-// Register copy: every thread issues kUnroll independent streaming loads, then
+// n / d through one multiply: m = floor(2^32 / d) + 1 (0 stands for d == 1).
+// Exact while n * d < 2^32, which the planner guarantees for every tile.
+__device__ __forceinline__ uint32_t fast_div(uint32_t n, uint32_t m)
+{
+    return m ? __umulhi(n, m) : n;
+}
+__device__ __forceinline__ uint32_t div_magic(uint32_t d)
+{
+    return d == 1u ? 0u : 0xFFFFFFFFu / d + 1u;  // for a power of two this is 2^32 / d, also exact
+}
+
+// Register copy: every thread issues U independent streaming loads, then
 // the matching stores.  Work item w = (tile, lc); a tile is ntok tokens x H
 // heads x row_bytes, addressed on each side by a token stride and a head
 // stride, so the head<->token transpose between the two pool layouts is a
 // permutation of whole rows and needs no shuffling inside a row.
-template <int W, bool CHECK>
-__global__ void __launch_bounds__(kMaxThreads)
+template <int W, int U, bool CHECK>
+__global__ void __launch_bounds__(max_threads(W, U))
 copy_tiles_kernel(const CopyParams p)
 {
     using V = typename VecT<W>::type;
@@ -55,6 +107,8 @@ copy_tiles_kernel(const CopyParams p)
                       p.dst.head_stride == p.row_bytes && p.dst.tok_stride == hrow;
     const int64_t n_work = (int64_t)p.n_tiles * p.n_lc;
     const uint32_t nthr = blockDim.x;
+    const uint32_t m_vpr = div_magic(vpr);
+    const uint32_t m_H = div_magic(H);
 
     for (int64_t w = blockIdx.x; w < n_work; w += gridDim.x) {
         int32_t ti, lci;
@@ -73,12 +127,14 @@ copy_tiles_kernel(const CopyParams p)
         const bool zero = t.src_off < 0;
         const uint32_t ntok = (uint32_t)t.ntok;
         const uint32_t nvec = ntok * H * vpr;
+        const uint32_t m_inner = head_inner ? m_H : div_magic(ntok);
+        const uint32_t inner = head_inner ? H : ntok;
 
-        for (uint32_t i0 = threadIdx.x; i0 < nvec; i0 += nthr * kUnroll) {
-            V v[kUnroll];
-            int64_t doff[kUnroll];
+        for (uint32_t i0 = threadIdx.x; i0 < nvec; i0 += nthr * U) {
+            V v[U];
+            int64_t doff[U];
 #pragma unroll
-            for (int k = 0; k < kUnroll; ++k) {
+            for (int k = 0; k < U; ++k) {
                 const uint32_t i = i0 + k * nthr;
                 v[k] = zero_vec<V>();
                 doff[k] = -1;
@@ -88,16 +144,12 @@ copy_tiles_kernel(const CopyParams p)
                         so = (int64_t)i * W;
                         dof = so;
                     } else {
-                        const uint32_t row = i / vpr;
+                        const uint32_t row = fast_div(i, m_vpr);
                         const uint32_t vv = i - row * vpr;
-                        uint32_t tk, hd;
-                        if (head_inner) {
-                            tk = row / H;
-                            hd = row - tk * H;
-                        } else {
-                            hd = row / ntok;
-                            tk = row - hd * ntok;
-                        }
+                        const uint32_t outer = fast_div(row, m_inner);
+                        const uint32_t in = row - outer * inner;
+                        const uint32_t tk = head_inner ? outer : in;
+                        const uint32_t hd = head_inner ? in : outer;
                         so = tk * p.src.tok_stride + hd * p.src.head_stride + (int64_t)vv * W;
                         dof = tk * p.dst.tok_stride + hd * p.dst.head_stride + (int64_t)vv * W;
                     }
@@ -110,26 +162,26 @@ copy_tiles_kernel(const CopyParams p)
                         }
                     }
                     doff[k] = dof;
-                    if (!zero) v[k] = __ldcs(reinterpret_cast<const V *>(p.src.base + so));
+                    if (!zero) v[k] = ld_stream<V>(p.src.base + so);
                 }
             }
 #pragma unroll
-            for (int k = 0; k < kUnroll; ++k)
-                if (doff[k] >= 0) __stcs(reinterpret_cast<V *>(p.dst.base + doff[k]), v[k]);
+            for (int k = 0; k < U; ++k)
+                if (doff[k] >= 0) st_stream<V>(p.dst.base + doff[k], v[k]);
         }
     }
 }
 
-template <int W>
-static cudaError_t launch_w(const CopyParams &p, const LaunchConfig &cfg, cudaStream_t stream)
+template <int W, int U>
+static cudaError_t launch_wu(const CopyParams &p, const LaunchConfig &cfg, cudaStream_t stream)
 {
     const int64_t n_work = (int64_t)p.n_tiles * p.n_lc;
     if (n_work <= 0) return cudaSuccess;
     int threads = cfg.threads;
-    if (threads > kMaxThreads) threads = kMaxThreads;
+    if (threads > max_threads(W, U)) threads = max_threads(W, U);
     if (threads < 32) threads = 32;
     threads = (threads / 32) * 32;
-    auto kern = cfg.check_bounds ? copy_tiles_kernel<W, true> : copy_tiles_kernel<W, false>;
+    auto kern = cfg.check_bounds ? copy_tiles_kernel<W, U, true> : copy_tiles_kernel<W, U, false>;
     int occ = 0;
     cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, threads, 0);
     if (e != cudaSuccess) return e;
@@ -141,14 +193,27 @@ static cudaError_t launch_w(const CopyParams &p, const LaunchConfig &cfg, cudaSt
     return cudaGetLastError();
 }
 
+template <int W>
+static cudaError_t launch_w(const CopyParams &p, const LaunchConfig &cfg, cudaStream_t stream)
+{
+    switch (cfg.unroll) {
+    case 1: return launch_wu<W, 1>(p, cfg, stream);
+    case 2: return launch_wu<W, 2>(p, cfg, stream);
+    case 4: return launch_wu<W, 4>(p, cfg, stream);
+    case 8: return launch_wu<W, 8>(p, cfg, stream);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
 cudaError_t launch_copy(const CopyParams &p, const LaunchConfig &cfg, cudaStream_t stream)
 {
     switch (cfg.vec_bytes) {
+    case 32: return launch_w<32>(p, cfg, stream);
     case 16: return launch_w<16>(p, cfg, stream);
-    case 8: return launch_w<8>(p, cfg, stream);
-    case 4: return launch_w<4>(p, cfg, stream);
-    case 2: return launch_w<2>(p, cfg, stream);
-    case 1: return launch_w<1>(p, cfg, stream);
+    case 8: return launch_wu<8, 4>(p, cfg, stream);
+    case 4: return launch_wu<4, 4>(p, cfg, stream);
+    case 2: return launch_wu<2, 4>(p, cfg, stream);
+    case 1: return launch_wu<1, 4>(p, cfg, stream);
     default: return cudaErrorInvalidValue;
     }
 }

@@ -24,7 +24,7 @@ def _gpu_lib():
     yield
     B.pdkv_tune("debug_bounds", 0)
     B.pdkv_tune("tile_bytes", 65536)
-    B.pdkv_tune("lc_fastest", 1)
+    B.pdkv_tune("lc_fastest", 0)
 
 
 def dev(a: np.ndarray):
@@ -116,7 +116,7 @@ def test_tile_size_and_work_order_do_not_change_the_result(oracle, tile_bytes, l
         check_all_ops(oracle, W.make_config(5, num_layers=1, n_req=30, src_block=32))
     finally:
         B.pdkv_tune("tile_bytes", 65536)
-        B.pdkv_tune("lc_fastest", 1)
+        B.pdkv_tune("lc_fastest", 0)
 
 
 @pytest.mark.parametrize("seed", range(16))
