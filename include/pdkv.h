@@ -196,8 +196,8 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream);
 
 /* Process-wide tunables, read when a plan is created or a call is launched:
  *   "tile_bytes"     target bytes moved per tile (default 65536)
- *   "ctas_per_sm"    persistent CTAs per SM (default 2)
- *   "threads"        threads per CTA, multiple of 32 (default 512; clamped to
+ *   "ctas_per_sm"    persistent CTAs per SM (default 4)
+ *   "threads"        threads per CTA, multiple of 32 (default 256; clamped to
  *                    what the register budget of the chosen variant allows)
  *   "unroll"         independent accesses in flight per thread: 1, 2, 4, 8 (default 1)
  *   "vec32"          1: use 32-byte accesses when rows and bases allow (default 1)

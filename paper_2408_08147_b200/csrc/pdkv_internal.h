@@ -56,8 +56,8 @@ cudaError_t launch_copy(const CopyParams &p, const LaunchConfig &cfg, cudaStream
 
 struct Tunables {
     int64_t tile_bytes = 65536;
-    int64_t ctas_per_sm = 2;
-    int64_t threads = 512;
+    int64_t ctas_per_sm = 4;
+    int64_t threads = 256;
     int64_t unroll = 1;
     int64_t vec32 = 1;
     int64_t lc_fastest = 0;
