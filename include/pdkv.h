@@ -73,7 +73,8 @@ enum pdkv_status {
     PDKV_ERR_BUFFER_TOO_SMALL = -4, /* contiguous buffer smaller than the plan needs */
     PDKV_ERR_CUDA = -5,             /* a CUDA runtime call failed */
     PDKV_ERR_DEVICE_BOUNDS = -6,    /* bounds-checked kernels refused an access (debug option) */
-    PDKV_ERR_NOMEM = -7             /* host allocation failed */
+    PDKV_ERR_NOMEM = -7,            /* host allocation failed */
+    PDKV_ERR_LIMIT = -8             /* batch larger than pdkv_transfer_noalloc's built-in scratch */
 };
 
 enum pdkv_op {
@@ -164,6 +165,45 @@ int pdkv_unpack(const pdkv_plan *plan, const void *buf, size_t buf_bytes,
  * pdkv_unpack, without materialising the buffer.  (No counterpart in the
  * paper, whose two pools sit on different devices.) */
 int pdkv_transfer(const pdkv_plan *plan, int layer_begin, int layer_end, void *stream);
+
+/* Fused transfer for callers that must not allocate device memory.  (The paper
+ * has no counterpart; this is a deployment convenience.)
+ *
+ * Who needs it: a serving engine that hands all of HBM to its own block
+ * allocator at start-up, a process running under a frozen memory pool, or code
+ * on a path where cudaMalloc's implicit device-wide synchronisation is not
+ * acceptable.  Such callers cannot use pdkv_plan_create(), which allocates the
+ * plan's tile list with cudaMalloc.  Here the tile list lives in a fixed array
+ * of PDKV_NOALLOC_SCRATCH_BYTES that is part of the library image: every GPU on
+ * which the library is used holds those bytes until the process exits, and no
+ * cudaMalloc, cudaFree or other allocating CUDA or framework routine is called
+ * (host-side bookkeeping uses ordinary heap memory).
+ *
+ * Arguments are those of pdkv_plan_create() + pdkv_transfer(): two pools, one
+ * batch (host arrays, read during the call), a layer range and a stream.  The
+ * decode pool receives exactly what pdkv_transfer() would write.
+ *
+ * Limits and caveats
+ *   - The batch may need at most PDKV_NOALLOC_MAX_TILES tiles (see
+ *     pdkv_plan_tiles(); roughly kept_tokens * H*D*E / "tile_bytes", plus one
+ *     per block boundary); beyond that PDKV_ERR_LIMIT is returned and nothing
+ *     is enqueued.  Raise "tile_bytes" or split the batch.
+ *   - The first call on each device looks up the device address of the scratch
+ *     array (with that device current).  Make that first call outside any
+ *     stream capture.
+ *   - Every call on a device reuses the same scratch, which still holds the
+ *     previous call's tiles; the call rewrites what it needs (including the
+ *     words that must start at zero) on `stream` before its kernel runs.  Two
+ *     calls whose GPU work can overlap (different streams without an ordering
+ *     between them) race on it: order them, or use plans.
+ *   - The tile list is copied from pageable host memory, so the call may block
+ *     until earlier work on `stream` has finished.
+ * Errors: INVALID_ARG, GEOMETRY, TABLE, LIMIT, CUDA, NOMEM. */
+#define PDKV_NOALLOC_MAX_TILES 32768
+#define PDKV_NOALLOC_SCRATCH_BYTES (256 + PDKV_NOALLOC_MAX_TILES * 24)
+int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
+                          const pdkv_batch_desc *batch, int layer_begin, int layer_end,
+                          void *stream);
 
 /* Baseline: the block-by-block transfer of Sec. 2.3 ("transfer one by one"),
  * one copy or one kernel launch per prefill block issued from a host loop.

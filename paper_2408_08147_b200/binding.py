@@ -27,6 +27,8 @@ PDKV_ERR_BUFFER_TOO_SMALL = -4
 PDKV_ERR_CUDA = -5
 PDKV_ERR_DEVICE_BOUNDS = -6
 PDKV_ERR_NOMEM = -7
+PDKV_ERR_LIMIT = -8
+PDKV_NOALLOC_MAX_TILES = 32768
 
 PDKV_OP_PACK = 0
 PDKV_OP_UNPACK = 1
@@ -36,7 +38,7 @@ PDKV_OP_BLOCKWISE = 3  # only for pdkv_plan_launches
 EXPORTS = (
     "pdkv_pool_bytes", "pdkv_pool_create", "pdkv_pool_destroy", "pdkv_plan_create",
     "pdkv_plan_destroy", "pdkv_plan_buffer", "pdkv_plan_traffic", "pdkv_pack", "pdkv_unpack",
-    "pdkv_transfer", "pdkv_transfer_blockwise", "pdkv_plan_launches", "pdkv_plan_tiles",
+    "pdkv_transfer", "pdkv_transfer_noalloc", "pdkv_transfer_blockwise", "pdkv_plan_launches", "pdkv_plan_tiles",
     "pdkv_plan_status", "pdkv_tune", "pdkv_tune_get", "pdkv_strerror",
 )
 
@@ -92,6 +94,7 @@ def lib() -> C.CDLL:
     L.pdkv_pack.argtypes = [vp, vp, C.c_size_t, C.c_int, C.c_int, vp]
     L.pdkv_unpack.argtypes = [vp, vp, C.c_size_t, C.c_int, C.c_int, vp]
     L.pdkv_transfer.argtypes = [vp, C.c_int, C.c_int, vp]
+    L.pdkv_transfer_noalloc.argtypes = [vp, vp, C.POINTER(pdkv_batch_desc), C.c_int, C.c_int, vp]
     L.pdkv_transfer_blockwise.argtypes = [vp, vp]
     L.pdkv_plan_launches.argtypes = [vp, C.c_int, C.POINTER(i64)]
     L.pdkv_plan_tiles.argtypes = [vp, C.c_int, C.POINTER(C.POINTER(pdkv_tile)), C.POINTER(i64)]
@@ -205,6 +208,19 @@ def pdkv_unpack(plan: int, buf_ptr: int, buf_bytes: int, layer_begin: int, layer
 def pdkv_transfer(plan: int, layer_begin: int, layer_end: int, stream: int = 0) -> None:
     _check(lib().pdkv_transfer(C.c_void_p(plan), layer_begin, layer_end, C.c_void_p(stream)),
            "pdkv_transfer")
+
+
+def pdkv_transfer_noalloc(src_pool: int, dst_pool: int, seq_len, src_tbl_off, src_tbl, dst_tbl_off,
+                          dst_tbl, dst_skip, layer_begin: int, layer_end: int,
+                          stream: int = 0) -> None:
+    """Fused transfer that allocates no device memory (no plan object): the
+    tile list goes into a fixed scratch array inside the library.  For callers
+    that may not call cudaMalloc; batches are limited to
+    ``PDKV_NOALLOC_MAX_TILES`` tiles, and overlapping calls race on the scratch."""
+    b = _BatchArrays(seq_len, src_tbl_off, src_tbl, dst_tbl_off, dst_tbl, dst_skip)
+    _check(lib().pdkv_transfer_noalloc(C.c_void_p(src_pool), C.c_void_p(dst_pool), C.byref(b.desc),
+                                       layer_begin, layer_end, C.c_void_p(stream)),
+           "pdkv_transfer_noalloc")
 
 
 def pdkv_transfer_blockwise(plan: int, stream: int = 0) -> None:

@@ -28,6 +28,7 @@ struct BlockGroup {     // one prefill block's share of the fused transfer (base
 };
 
 thread_local std::string g_cuda_msg;
+thread_local bool g_host_only_plan = false;  // set only around pdkv::create_host_plan()
 
 int cuda_fail(cudaError_t e, const char *what)
 {
@@ -271,6 +272,33 @@ Tunables &tunables()
 }
 }  // namespace pdkv
 
+namespace pdkv {
+
+int create_host_plan(const pdkv_pool *src, const pdkv_pool *dst, const pdkv_batch_desc *batch,
+                     pdkv_plan **out)
+{
+    g_host_only_plan = true;
+    const int rc = pdkv_plan_create(src, dst, 0, batch, nullptr, out);
+    g_host_only_plan = false;
+    return rc;
+}
+
+void describe_transfer(const pdkv_plan *plan, Side *src, Side *dst, int *H, int *row_bytes,
+                       int *vec_bytes, int *num_layers, int *device)
+{
+    *src = pool_side(plan->src, plan->row_bytes, plan->hrow_bytes);
+    *dst = pool_side(plan->dst, plan->row_bytes, plan->hrow_bytes);
+    *H = plan->H;
+    *row_bytes = (int)plan->row_bytes;
+    *vec_bytes = plan->vec_bytes;
+    *num_layers = plan->L;
+    *device = plan->device;
+}
+
+int report_cuda_error(cudaError_t e, const char *what) { return cuda_fail(e, what); }
+
+}  // namespace pdkv
+
 extern "C" {
 
 size_t pdkv_pool_bytes(const pdkv_pool_desc *d)
@@ -429,7 +457,7 @@ int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip_gr
         for (int op = 0; op < 3; ++op)
             if (pl->tiles[op].size() > (size_t)INT32_MAX) return PDKV_ERR_INVALID_ARG;
 
-        if (pdkv::tunables().dry_run) {  // host-only plan: tile lists can be inspected, nothing can launch
+        if (pdkv::tunables().dry_run || g_host_only_plan) {  // host-only plan: tile lists can be inspected, nothing can launch
             hold.p = nullptr;
             *out = pl;
             return PDKV_OK;
@@ -653,6 +681,7 @@ const char *pdkv_strerror(int status)
     case PDKV_ERR_CUDA: return g_cuda_msg.empty() ? "CUDA error" : g_cuda_msg.c_str();
     case PDKV_ERR_DEVICE_BOUNDS: return g_cuda_msg.empty() ? "device bounds check refused an access" : g_cuda_msg.c_str();
     case PDKV_ERR_NOMEM: return "out of host memory";
+    case PDKV_ERR_LIMIT: return "batch exceeds the built-in scratch of the no-allocation entry point";
     default: return "unknown status";
     }
 }

@@ -67,4 +67,12 @@ struct Tunables {
 };
 Tunables &tunables();
 
+// Used by the no-allocation entry point (its own translation unit).
+// A host-only plan: validated batch and tile lists, no CUDA call, nothing on the device.
+int create_host_plan(const pdkv_pool *src, const pdkv_pool *dst, const pdkv_batch_desc *batch,
+                     pdkv_plan **out);
+void describe_transfer(const pdkv_plan *plan, Side *src, Side *dst, int *H, int *row_bytes,
+                       int *vec_bytes, int *num_layers, int *device);
+int report_cuda_error(cudaError_t e, const char *what);
+
 }  // namespace pdkv

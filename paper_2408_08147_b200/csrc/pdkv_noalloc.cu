@@ -1,0 +1,121 @@
+// Fused transfer without any device allocation: the tile list that the copy
+// kernel walks is staged in a fixed device array that ships with the library.
+//
+// Intended for callers that may not call cudaMalloc: engines that gave all of
+// HBM to their own block allocator, processes under a frozen memory pool, or
+// latency paths that cannot afford cudaMalloc's device-wide synchronisation.
+#include <mutex>
+
+#include "pdkv_internal.h"
+
+namespace {
+
+constexpr size_t kHeaderBytes = 256;  // status words of the kernels, cleared by every call
+static_assert(sizeof(pdkv::Tile) == 24, "PDKV_NOALLOC_SCRATCH_BYTES assumes 24-byte tiles");
+static_assert(PDKV_NOALLOC_SCRATCH_BYTES == kHeaderBytes + PDKV_NOALLOC_MAX_TILES * sizeof(pdkv::Tile),
+              "scratch size and tile limit must agree");
+
+// Scratch shared by every call on a device: [status words][tile list].  Each
+// GPU that loads this library keeps its own copy until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[PDKV_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+struct DeviceSlot {
+    unsigned char *scratch = nullptr;  // device address of g_noalloc_scratch on that device
+    int sm_count = 0;
+};
+DeviceSlot g_slots[kMaxDevices];
+std::mutex g_slots_mutex;
+
+// Once per device, with that device current: the array's name is only a
+// host-side handle, so the kernel must be given the address looked up here.
+cudaError_t device_slot(int device, DeviceSlot *out)
+{
+    std::lock_guard<std::mutex> lock(g_slots_mutex);
+    DeviceSlot &s = g_slots[device];
+    if (!s.scratch) {
+        void *ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+        if (e != cudaSuccess) return e;
+        int sms = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+        if (e != cudaSuccess) return e;
+        s.sm_count = sms;
+        s.scratch = static_cast<unsigned char *>(ptr);
+    }
+    *out = s;
+    return cudaSuccess;
+}
+
+struct PlanHolder {
+    pdkv_plan *p = nullptr;
+    ~PlanHolder() { if (p) pdkv_plan_destroy(p); }
+};
+
+}  // namespace
+
+extern "C" int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
+                                     const pdkv_batch_desc *batch, int layer_begin, int layer_end,
+                                     void *stream)
+{
+    if (!src || !dst || !batch) return PDKV_ERR_INVALID_ARG;
+    PlanHolder plan;  // host memory only: validated batch and its tile lists
+    int rc = pdkv::create_host_plan(src, dst, batch, &plan.p);
+    if (rc != PDKV_OK) return rc;
+
+    pdkv::CopyParams p;
+    int vec_bytes = 16, num_layers = 0, device = 0, H = 0, row_bytes = 0;
+    pdkv::describe_transfer(plan.p, &p.src, &p.dst, &H, &row_bytes, &vec_bytes, &num_layers, &device);
+    if (layer_begin < 0 || layer_begin > layer_end || layer_end > num_layers) return PDKV_ERR_INVALID_ARG;
+    if (device < 0 || device >= kMaxDevices) return PDKV_ERR_INVALID_ARG;
+
+    const pdkv_tile *tiles = nullptr;
+    int64_t n_tiles = 0;
+    rc = pdkv_plan_tiles(plan.p, PDKV_OP_TRANSFER, &tiles, &n_tiles);
+    if (rc != PDKV_OK) return rc;
+    if (n_tiles > PDKV_NOALLOC_MAX_TILES) return PDKV_ERR_LIMIT;
+    if (n_tiles == 0 || layer_begin == layer_end) return PDKV_OK;
+
+    int prev = -1;
+    cudaError_t e = cudaGetDevice(&prev);
+    if (e != cudaSuccess) return pdkv::report_cuda_error(e, "cudaGetDevice");
+    if (prev != device && (e = cudaSetDevice(device)) != cudaSuccess)
+        return pdkv::report_cuda_error(e, "cudaSetDevice");
+
+    rc = PDKV_OK;
+    DeviceSlot slot;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((e = device_slot(device, &slot)) != cudaSuccess) {
+        rc = pdkv::report_cuda_error(e, "cudaGetSymbolAddress");
+    } else if ((e = cudaMemsetAsync(slot.scratch, 0, kHeaderBytes, st)) != cudaSuccess) {
+        rc = pdkv::report_cuda_error(e, "cudaMemsetAsync");
+    } else if ((e = cudaMemcpyAsync(slot.scratch + kHeaderBytes, tiles, (size_t)n_tiles * sizeof(pdkv::Tile),
+                                    cudaMemcpyHostToDevice, st)) != cudaSuccess) {
+        rc = pdkv::report_cuda_error(e, "cudaMemcpyAsync");
+    } else {
+        const pdkv::Tunables &t = pdkv::tunables();
+        p.tiles = reinterpret_cast<const pdkv::Tile *>(slot.scratch + kHeaderBytes);
+        p.tile_begin = 0;
+        p.n_tiles = (int32_t)n_tiles;
+        p.lc_begin = 2 * layer_begin;
+        p.n_lc = 2 * (layer_end - layer_begin);
+        p.H = H;
+        p.row_bytes = row_bytes;
+        p.lc_fastest = (int32_t)t.lc_fastest;
+        p.status = reinterpret_cast<unsigned long long *>(slot.scratch);
+        pdkv::LaunchConfig cfg;
+        cfg.vec_bytes = vec_bytes;
+        if (vec_bytes == 16 && t.vec32 && row_bytes % 32 == 0 &&
+            ((reinterpret_cast<uintptr_t>(p.src.base) | reinterpret_cast<uintptr_t>(p.dst.base)) & 31u) == 0)
+            cfg.vec_bytes = 32;
+        cfg.unroll = (int)t.unroll;
+        cfg.threads = (int)t.threads;
+        cfg.ctas_per_sm = (int)t.ctas_per_sm;
+        cfg.sm_count = slot.sm_count;
+        cfg.variant = 0;
+        cfg.check_bounds = false;
+        if ((e = pdkv::launch_copy(p, cfg, st)) != cudaSuccess) rc = pdkv::report_cuda_error(e, "kernel launch");
+    }
+    if (prev != device) cudaSetDevice(prev);
+    return rc;
+}
