@@ -426,7 +426,7 @@ def main_arm(args):
            "ops": per_op, "roofline": roofline, "gpu_launches": launches_per_step * args.steps,
            "sanity_check": "ok" if ok else "MISMATCH", "clocks": clk.summary()}
 
-    if rank == 0 and not args.no_extras:
+    if rank == 0 and not args.no_extras and not args.no_blockwise:
         # block-by-block baseline (Sec. 2.3 "transfer one by one"): same result, host loop
         n_blk = sess.launches(B.PDKV_OP_BLOCKWISE)
         reps = max(1, min(5, args.steps))
@@ -445,7 +445,7 @@ def main_arm(args):
                                      "fused_speedup": bw_ms / op_ms["fused"]}
 
     # end to end: pinned host pools, H2D of the prefill pool, plan, the three calls, D2H of the decode pool
-    if not args.no_extras:
+    if not args.no_extras and not args.no_e2e:
         try:
             out["e2e"] = e2e_leg(args, w, src_t, dst_t, buf_t, stream, step_bytes, torch, B, TransferSession, dev)
         except Exception as e:  # pragma: no cover
@@ -527,6 +527,8 @@ def parse():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-extras", action="store_true", help="skip baseline, e2e and CPU legs")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-blockwise", action="store_true")
     return ap.parse_args()
 
 
