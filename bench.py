@@ -34,8 +34,12 @@ KERNEL_SOURCE = os.path.join(ROOT, "paper_2408_08147_b200", "csrc", "pdkv_kernel
 
 # DRAM traffic per launch from ncu (dram__bytes_read.sum + dram__bytes_write.sum),
 # keyed by (workload, op); valid only while the kernel source hashes to KERNEL_SHA.
-NCU_TRAFFIC: dict = {}
-NCU_KERNEL_SHA = ""
+# Captured on a 1/8-size case (4 of 32 requests; profiles/copy_tiles_kernel_config2_small_ncu_full.md)
+# and scaled by 8: traffic is proportional to the tokens moved (read 1.0738 GB + write 1.031 GB
+# per 2.1475 GB algorithmic).
+NCU_TRAFFIC: dict = {(2, "pack"): 8 * (1.074010e9 + 1.029354e9), (2, "unpack"): 8 * (1.073795e9 + 1.031753e9),
+                     (2, "fused"): 8 * (1.073809e9 + 1.031127e9)}
+NCU_KERNEL_SHA = "cba665c32a89e1e1"
 
 
 def log(*a):
