@@ -358,6 +358,7 @@ def main_arm(args):
         kw["src_layout"], kw["dst_layout"] = ("AB".index(args.layouts[0]), "AB".index(args.layouts[1]))
     w = W.make_config(args.config, **kw)
     src_t, dst_t = alloc_pools(w, torch, seed_offset=rank)
+    torch.cuda.synchronize()          # the fills ran on torch's stream, the library gets its own
     stream = torch.cuda.Stream()
     sess = TransferSession(w.src, src_t, w.dst, dst_t, w.batch, stream.cuda_stream)
     buf_t = torch.empty(max(sess.buffer_bytes, 16), dtype=torch.uint8, device=dev)

@@ -1,0 +1,141 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration the
+benchmark times (library defaults).  Pools of 8-50 GiB cannot be replayed on the
+CPU checker in full, so a seeded sample of requests is checked bit for bit:
+each sampled request becomes a self-contained sub-problem (its blocks gathered
+out of both pools), the checker computes buffer and decode blocks for it, and
+the GPU's bytes for that request must be identical.  Bytes nobody may touch
+(resident decode blocks, the buffer's slack) are compared with the sentinel."""
+import numpy as np
+import pytest
+
+from paper_2408_08147_b200 import binding as B
+from paper_2408_08147_b200 import workloads as W
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+SENT = W.SENTINEL_U16
+SLACK = 4096
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _defaults():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    B.lib()
+    B.pdkv_tune("dry_run", 0)
+    B.pdkv_tune("debug_bounds", 0)
+    yield
+    torch.cuda.empty_cache()
+
+
+def _sentinel_fill(t):
+    t.view(torch.int16).fill_(SENT)
+    torch.cuda.synchronize()        # the library runs on its own stream
+
+
+def _np16(t):
+    return t.cpu().numpy().view(np.uint16)
+
+
+def run_fullsize(oracle, w, n_sample, seed):
+    from paper_2408_08147_b200.session import TransferSession
+
+    import gc
+
+    gc.collect()
+    torch.cuda.empty_cache()        # earlier tests' pools sit in torch's cache, not in the driver's free list
+    need = w.src.num_bytes() + 2 * w.dst.num_bytes()
+    free, _ = torch.cuda.mem_get_info()
+    if need * 1.1 > free:
+        pytest.skip(f"needs {need >> 30} GiB of device memory")
+    b = w.batch
+    rng = np.random.default_rng(seed)
+    sample = sorted({0, b.n_req - 1, *rng.integers(0, b.n_req, size=max(0, n_sample - 2)).tolist()})
+
+    src_t = torch.empty(w.src.num_bytes(), dtype=torch.uint8, device="cuda")
+    W.fill_pool_torch(src_t, w.seed)
+    dst_t = torch.empty(w.dst.num_bytes(), dtype=torch.uint8, device="cuda")
+    _sentinel_fill(dst_t)
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    G = w.dst.block_tokens
+
+    with TransferSession(w.src, src_t, w.dst, dst_t, b, stream.cuda_stream) as s:
+        assert s.buffer_bytes == sum(s.traffic(B.PDKV_OP_PACK)) // 2
+        buf_t = torch.empty(s.buffer_bytes + SLACK, dtype=torch.uint8, device="cuda")
+        _sentinel_fill(buf_t)
+
+        # expected bytes of every sampled request, from the checker
+        expect = {}
+        for r in sample:
+            sub, s_ids, d_ids = W.compact_subproblem(w, [r])
+            sub_src = _np16(W.gather_blocks(src_t.view(torch.int16), w.src, s_ids))
+            want_buf = np.zeros(oracle.buffer_elems(sub.batch, G, sub.src), np.uint16)
+            oracle.pack(sub.src, sub_src, sub.batch, G, want_buf)
+            want_dst = W.sentinel_pool_numpy(sub.dst)
+            oracle.transfer(sub.src, sub_src, sub.dst, want_dst, sub.batch)
+            expect[r] = (want_buf, want_dst, d_ids)
+            assert want_buf.size * 2 == s.request_offsets[r + 1] - s.request_offsets[r]
+
+        def check_dst(what):
+            for r, (_, want_dst, d_ids) in expect.items():
+                got = _np16(W.gather_blocks(dst_t.view(torch.int16), w.dst, d_ids))
+                assert np.array_equal(got, want_dst), f"{what}: request {r}"
+
+        s.pack(buf_t)
+        torch.cuda.synchronize()
+        for r, (want_buf, _, _) in expect.items():
+            a, z = int(s.request_offsets[r]), int(s.request_offsets[r + 1])
+            assert np.array_equal(_np16(buf_t[a:z]), want_buf), f"pack: request {r}"
+        assert bool((buf_t[s.buffer_bytes:].view(torch.int16) == SENT).all()), "pack wrote past the buffer"
+
+        s.unpack(buf_t)
+        torch.cuda.synchronize()
+        check_dst("unpack")
+
+        _sentinel_fill(dst_t)
+        s.transfer()
+        torch.cuda.synchronize()
+        check_dst("fused")
+
+        # resident (skipped) decode blocks keep the sentinel
+        if b.dst_skip is not None:
+            nblk = -(-b.seq_len.astype(np.int64) // G)
+            ids = np.concatenate([b.dst_tbl[b.dst_tbl_off[r]:b.dst_tbl_off[r] + nblk[r]]
+                                  [b.dst_skip[b.dst_tbl_off[r]:b.dst_tbl_off[r] + nblk[r]] != 0]
+                                  for r in range(b.n_req)])
+            assert ids.size > 0
+            for i in range(0, ids.size, 64):
+                blk = W.gather_blocks(dst_t.view(torch.int16), w.dst, ids[i:i + 64])
+                assert bool((blk == SENT).all()), "a resident decode block was written"
+
+        _sentinel_fill(dst_t)
+        s.transfer_blockwise()
+        torch.cuda.synchronize()
+        check_dst("block-by-block baseline")
+    del src_t, dst_t, buf_t, s
+    torch.cuda.empty_cache()
+
+
+def test_config2_full_size_same_layout(oracle):
+    run_fullsize(oracle, W.make_config(2), n_sample=4, seed=2)
+
+
+def test_config2_full_size_layer_major_both_sides(oracle):
+    run_fullsize(oracle, W.make_config(2, src_layout=W.LAYER_MAJOR), n_sample=3, seed=22)
+
+
+def test_config3_full_size_reblocking(oracle):
+    run_fullsize(oracle, W.make_config(3), n_sample=5, seed=3)
+
+
+def test_config4_full_size_70b_fragmented(oracle):
+    w = W.make_config(4)
+    assert w.src.num_elems() > 2 ** 32          # offsets beyond 32 bits
+    run_fullsize(oracle, w, n_sample=2, seed=4)
+
+
+@pytest.mark.parametrize("src_block", [16, 256])
+def test_config5_full_size_skip_mask(oracle, src_block):
+    run_fullsize(oracle, W.make_config(5, src_block=src_block), n_sample=8, seed=5 + src_block)

@@ -67,17 +67,20 @@ def check_all_ops(oracle, w, *, layers=None, elem_dtype=np.uint16, side_stream=F
         assert np.array_equal(host(src_t, elem_dtype), src), "pack wrote the source pool"
 
         fb_t = dev(full_buf)
+        torch.cuda.synchronize()
         s.unpack(fb_t, layers)
         s.status()
         assert np.array_equal(host(dst_t, elem_dtype), want_dst), "unpack"
 
         dst_t.copy_(dev(sent))
+        torch.cuda.synchronize()
         s.transfer(layers)
         s.status()
         assert np.array_equal(host(dst_t, elem_dtype), want_dst), "fused transfer"
 
         if blockwise and layers is None:
             dst_t.copy_(dev(sent))
+            torch.cuda.synchronize()
             s.transfer_blockwise()
             s.status()
             assert np.array_equal(host(dst_t, elem_dtype), want_dst), "block-by-block baseline"
@@ -202,6 +205,7 @@ def test_per_layer_calls_equal_whole_model(oracle):
         torch.cuda.synchronize()
         assert np.array_equal(host(dst_t), want)
         dst_t.copy_(dev(sent))
+        torch.cuda.synchronize()
         for l in reversed(range(4)):
             s.transfer((l, l + 1))
         s.status()
