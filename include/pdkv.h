@@ -243,6 +243,8 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream);
  *   "vec32"          1: use 32-byte accesses when rows and bases allow (default 1)
  *   "lc_fastest"     1: consecutive work items walk the (layer, K/V) strips of
  *                    one tile; 0: they walk the tiles of one strip (default 0)
+ *   "chunked"        1: each CTA takes one contiguous run of work items instead
+ *                    of every gridDim-th one (default 0)
  *   "debug_bounds"   1: kernels range-check every access and skip bad ones
  *   "variant"        0: register copy, 1: bulk async copy through shared memory
  *   "dry_run"        1: pdkv_plan_create builds host-only plans (no CUDA call is

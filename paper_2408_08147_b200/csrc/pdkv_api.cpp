@@ -241,6 +241,7 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     p.H = pl->H;
     p.row_bytes = (int32_t)pl->row_bytes;
     p.lc_fastest = (int32_t)pdkv::tunables().lc_fastest;
+    p.chunked = (int32_t)pdkv::tunables().chunked;
     p.status = pl->dev_status;
     pdkv::LaunchConfig cfg;
     cfg.vec_bytes = pl->vec_bytes;
@@ -645,6 +646,7 @@ int pdkv_tune(const char *key, int64_t value)
     else if (k == "unroll" && (value == 1 || value == 2 || value == 4 || value == 8)) t.unroll = value;
     else if (k == "vec32" && (value == 0 || value == 1)) t.vec32 = value;
     else if (k == "lc_fastest" && (value == 0 || value == 1)) t.lc_fastest = value;
+    else if (k == "chunked" && (value == 0 || value == 1)) t.chunked = value;
     else if (k == "debug_bounds" && (value == 0 || value == 1)) t.debug_bounds = value;
     else if (k == "variant" && value >= 0 && value <= 1) t.variant = value;
     else if (k == "dry_run" && (value == 0 || value == 1)) t.dry_run = value;
@@ -663,6 +665,7 @@ int pdkv_tune_get(const char *key, int64_t *value)
     else if (k == "unroll") *value = t.unroll;
     else if (k == "vec32") *value = t.vec32;
     else if (k == "lc_fastest") *value = t.lc_fastest;
+    else if (k == "chunked") *value = t.chunked;
     else if (k == "debug_bounds") *value = t.debug_bounds;
     else if (k == "variant") *value = t.variant;
     else if (k == "dry_run") *value = t.dry_run;

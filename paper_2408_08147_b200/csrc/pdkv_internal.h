@@ -38,6 +38,7 @@ struct CopyParams {
     int32_t H;
     int32_t row_bytes;   // D * E
     int32_t lc_fastest;
+    int32_t chunked;     // 1: each CTA takes one contiguous run of work items
     unsigned long long *status;  // [0] != 0: an access was refused; [1] offending offset
 };
 
@@ -61,6 +62,7 @@ struct Tunables {
     int64_t unroll = 1;
     int64_t vec32 = 1;
     int64_t lc_fastest = 0;
+    int64_t chunked = 0;
     int64_t debug_bounds = 0;
     int64_t variant = 0;
     int64_t dry_run = 0;

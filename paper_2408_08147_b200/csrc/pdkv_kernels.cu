@@ -110,16 +110,45 @@ copy_tiles_kernel(const CopyParams p)
     const uint32_t m_vpr = div_magic(vpr);
     const uint32_t m_H = div_magic(H);
 
-    for (int64_t w = blockIdx.x; w < n_work; w += gridDim.x) {
-        int32_t ti, lci;
+    // Work items of this CTA: either every gridDim-th item (the CTAs sweep the
+    // batch as one moving window) or one contiguous run per CTA.
+    int64_t w, w_end, w_step;
+    if (p.chunked) {
+        const int64_t per = (n_work + gridDim.x - 1) / gridDim.x;
+        w = (int64_t)blockIdx.x * per;
+        w_end = w + per < n_work ? w + per : n_work;
+        w_step = 1;
+    } else {
+        w = blockIdx.x;
+        w_end = n_work;
+        w_step = gridDim.x;
+    }
+    auto split = [&](int64_t x, int32_t &ti, int32_t &lci) {
         if (p.lc_fastest) {
-            ti = (int32_t)(w / p.n_lc);
-            lci = (int32_t)(w - (int64_t)ti * p.n_lc);
+            ti = (int32_t)(x / p.n_lc);
+            lci = (int32_t)(x - (int64_t)ti * p.n_lc);
         } else {
-            lci = (int32_t)(w / p.n_tiles);
-            ti = (int32_t)(w - (int64_t)lci * p.n_tiles);
+            lci = (int32_t)(x / p.n_tiles);
+            ti = (int32_t)(x - (int64_t)lci * p.n_tiles);
         }
-        const Tile t = p.tiles[p.tile_begin + ti];
+    };
+    // The next item's tile record is fetched while the current one is being
+    // copied, so its latency is off the critical path between two tiles.
+    Tile t_next = {};
+    int32_t lci_next = 0;
+    if (w < w_end) {
+        int32_t ti;
+        split(w, ti, lci_next);
+        t_next = p.tiles[p.tile_begin + ti];
+    }
+    for (; w < w_end; w += w_step) {
+        const Tile t = t_next;
+        const int32_t lci = lci_next;
+        if (w + w_step < w_end) {
+            int32_t ti;
+            split(w + w_step, ti, lci_next);
+            t_next = p.tiles[p.tile_begin + ti];
+        }
         const int64_t lc = p.lc_begin + lci;
         const int64_t buf_lc = (int64_t)t.n_kept * hrow;
         const int64_t s_base = t.src_off + lc * (p.src.lc_stride >= 0 ? p.src.lc_stride : buf_lc);
