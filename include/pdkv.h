@@ -229,9 +229,10 @@ typedef struct {
 /* Host copy of the tile list of `op`, owned by the plan. */
 int pdkv_plan_tiles(const pdkv_plan *plan, int op, const pdkv_tile **tiles, int64_t *n_tiles);
 
-/* Synchronise `stream` and report the bounds-check word of the plan: PDKV_OK,
- * PDKV_ERR_DEVICE_BOUNDS (an access was refused and skipped) or
- * PDKV_ERR_CUDA.  Only meaningful with the "debug_bounds" option set. */
+/* Synchronise `stream` and report the plan's device status word: PDKV_OK,
+ * PDKV_ERR_DEVICE_BOUNDS (with "debug_bounds": an access was refused and
+ * skipped; with "variant" 1: a bounded wait on a bulk copy gave up and the
+ * kernel returned early) or PDKV_ERR_CUDA. */
 int pdkv_plan_status(const pdkv_plan *plan, void *stream);
 
 /* Process-wide tunables, read when a plan is created or a call is launched:
@@ -246,7 +247,11 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream);
  *   "chunked"        1: each CTA takes one contiguous run of work items instead
  *                    of every gridDim-th one (default 0)
  *   "debug_bounds"   1: kernels range-check every access and skip bad ones
- *   "variant"        0: register copy, 1: bulk async copy through shared memory
+ *   "variant"        0: register copy (default); 1: bulk async copies (TMA) through
+ *                    shared memory, one warp per CTA; used when rows are multiples
+ *                    of 16 bytes and a tile fits a stage, else variant 0 runs
+ *   "stages"         variant 1: shared-memory stages per CTA, 2..16 (default 3);
+ *                    stages x "tile_bytes" must fit in 220 KiB
  *   "dry_run"        1: pdkv_plan_create builds host-only plans (no CUDA call is
  *                    made; the plan can be inspected but not launched)
  * Unknown keys or out-of-range values give INVALID_ARG. */

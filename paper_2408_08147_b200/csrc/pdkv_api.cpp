@@ -91,6 +91,7 @@ struct pdkv_plan {
     void *dev_mem = nullptr;
     unsigned long long *dev_status = nullptr;
     int vec_bytes = 16;
+    int64_t max_tile_bytes = 0;
     int sm_count = 1;
     int lc_fastest = 1;
 };
@@ -254,7 +255,15 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     cfg.sm_count = pl->sm_count;
     cfg.variant = (int)pdkv::tunables().variant;
     cfg.check_bounds = pdkv::tunables().debug_bounds != 0;
-    cudaError_t e = pdkv::launch_copy(p, cfg, stream);
+    cfg.stages = (int)pdkv::tunables().stages;
+    cfg.max_tile_bytes = pl->max_tile_bytes;
+    cudaError_t e;
+    if (cfg.variant == 1 && pdkv::bulk_supported(cfg, p.row_bytes)) {
+        cfg.vec_bytes = 16;
+        e = pdkv::launch_bulk(p, cfg, stream);
+    } else {
+        e = pdkv::launch_copy(p, cfg, stream);
+    }
     if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
     return PDKV_OK;
 }
@@ -455,8 +464,11 @@ int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip_gr
         if (src) build_tiles(*pl, PDKV_OP_PACK, *batch, cap_tok);
         if (dst) build_tiles(*pl, PDKV_OP_UNPACK, *batch, cap_tok);
         if (src && dst) build_tiles(*pl, PDKV_OP_TRANSFER, *batch, cap_tok);
-        for (int op = 0; op < 3; ++op)
+        for (int op = 0; op < 3; ++op) {
             if (pl->tiles[op].size() > (size_t)INT32_MAX) return PDKV_ERR_INVALID_ARG;
+            for (const Tile &t : pl->tiles[op])
+                pl->max_tile_bytes = std::max<int64_t>(pl->max_tile_bytes, t.ntok * pl->hrow_bytes);
+        }
 
         if (pdkv::tunables().dry_run || g_host_only_plan) {  // host-only plan: tile lists can be inspected, nothing can launch
             hold.p = nullptr;
@@ -628,7 +640,10 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream)
     if (e != cudaSuccess) return cuda_fail(e, "status read");
     if (word[0]) {
         char msg[96];
-        std::snprintf(msg, sizeof(msg), "refused access at byte offset %lld", (long long)word[1]);
+        if (word[0] == 2)
+            std::snprintf(msg, sizeof(msg), "a bulk-copy wait gave up at work item %lld", (long long)word[1]);
+        else
+            std::snprintf(msg, sizeof(msg), "refused access at byte offset %lld", (long long)word[1]);
         g_cuda_msg = msg;
         return PDKV_ERR_DEVICE_BOUNDS;
     }
@@ -649,6 +664,7 @@ int pdkv_tune(const char *key, int64_t value)
     else if (k == "chunked" && (value == 0 || value == 1)) t.chunked = value;
     else if (k == "debug_bounds" && (value == 0 || value == 1)) t.debug_bounds = value;
     else if (k == "variant" && value >= 0 && value <= 1) t.variant = value;
+    else if (k == "stages" && value >= 2 && value <= 16) t.stages = value;
     else if (k == "dry_run" && (value == 0 || value == 1)) t.dry_run = value;
     else return PDKV_ERR_INVALID_ARG;
     return PDKV_OK;
@@ -668,6 +684,7 @@ int pdkv_tune_get(const char *key, int64_t *value)
     else if (k == "chunked") *value = t.chunked;
     else if (k == "debug_bounds") *value = t.debug_bounds;
     else if (k == "variant") *value = t.variant;
+    else if (k == "stages") *value = t.stages;
     else if (k == "dry_run") *value = t.dry_run;
     else return PDKV_ERR_INVALID_ARG;
     return PDKV_OK;

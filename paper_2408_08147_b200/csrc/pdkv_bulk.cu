@@ -1,0 +1,275 @@
+// Bulk-copy variant of the tile copy: one warp per CTA drives the TMA unit
+// (cp.async.bulk global -> shared -> global, mbarrier-tracked) through a ring
+// of shared-memory stages, one tile per stage.  No data passes through
+// registers, so the kernel occupies one warp and a few registers per CTA: this
+// is the "operator" form of RecvScatter that leaves the SMs' issue slots and
+// register file to whatever else runs in the stream (Sec. 3.5, "does not
+// interrupt the computation of other operators").
+//
+// A tile is staged in *destination order*.  Towards a head-major pool that is
+// [head][token][row]: the H stores are contiguous runs of ntok*ROW bytes and
+// the loads are one bulk copy per row when the source is token-major (the
+// head<->token transpose happens in the load addresses), or one per head when
+// the source is head-major too.  Towards a token-major side (block-major pool
+// or the contiguous buffer) the stage is [token][head][row] and the store is a
+// single bulk copy.
+//
+// Every wait is bounded: after kSpinLimit failed polls the warp records an
+// error word, drains its own stores and returns.
+#include "pdkv_internal.h"
+
+namespace pdkv {
+
+namespace {
+
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int kBarrierBytes = 128;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *b, int count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect(uint64_t *b, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *b)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *b, uint32_t phase)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(smem_u32(b)), "r"(phase)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_g2s(void *sdst, const void *gsrc, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(sdst)),
+                 "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_s2g(void *gdst, const void *ssrc, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(ssrc)),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t fast_div(uint32_t n, uint32_t m) { return m ? __umulhi(n, m) : n; }
+__device__ __forceinline__ uint32_t div_magic(uint32_t d) { return d == 1u ? 0u : 0xFFFFFFFFu / d + 1u; }
+
+struct Item {
+    int64_t s_base, d_base;
+    uint32_t ntok;
+    bool zero;
+};
+
+}  // namespace
+
+__global__ void __launch_bounds__(32) bulk_tiles_kernel(const CopyParams p, const int stages, const uint32_t stage_bytes)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem);
+    unsigned char *data = smem + kBarrierBytes;
+    const uint32_t lane = threadIdx.x;
+    const uint32_t H = (uint32_t)p.H;
+    const uint32_t row = (uint32_t)p.row_bytes;
+    const int64_t hrow = (int64_t)p.H * p.row_bytes;
+    const bool src_tok_major = p.src.tok_stride >= p.src.head_stride;
+    const bool dst_tok_major = p.dst.tok_stride >= p.dst.head_stride;
+    const bool src_flat = p.src.head_stride == p.row_bytes && p.src.tok_stride == hrow;
+    const bool dst_flat = p.dst.head_stride == p.row_bytes && p.dst.tok_stride == hrow;
+    const uint32_t m_H = div_magic(H);
+
+    if (lane == 0) {
+        for (int i = 0; i < stages; ++i) mbar_init(full + i, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+
+    const int64_t n_work = (int64_t)p.n_tiles * p.n_lc;
+    int64_t first, step, n_mine;
+    if (p.chunked) {
+        const int64_t per = (n_work + gridDim.x - 1) / gridDim.x;
+        first = (int64_t)blockIdx.x * per;
+        const int64_t end = first + per < n_work ? first + per : n_work;
+        n_mine = end > first ? end - first : 0;
+        step = 1;
+    } else {
+        first = blockIdx.x;
+        step = gridDim.x;
+        n_mine = n_work > first ? (n_work - first + step - 1) / step : 0;
+    }
+
+    auto item = [&](int64_t j) {
+        const int64_t w = first + j * step;
+        int32_t ti, lci;
+        if (p.lc_fastest) {
+            ti = (int32_t)(w / p.n_lc);
+            lci = (int32_t)(w - (int64_t)ti * p.n_lc);
+        } else {
+            lci = (int32_t)(w / p.n_tiles);
+            ti = (int32_t)(w - (int64_t)lci * p.n_tiles);
+        }
+        const Tile t = p.tiles[p.tile_begin + ti];
+        const int64_t lc = p.lc_begin + lci;
+        const int64_t buf_lc = (int64_t)t.n_kept * hrow;
+        Item it;
+        it.s_base = t.src_off + lc * (p.src.lc_stride >= 0 ? p.src.lc_stride : buf_lc);
+        it.d_base = t.dst_off + lc * (p.dst.lc_stride >= 0 ? p.dst.lc_stride : buf_lc);
+        it.ntok = (uint32_t)t.ntok;
+        it.zero = t.src_off < 0;
+        return it;
+    };
+
+    // Fill stage (j % stages) with item j, laid out in destination order.
+    auto issue_load = [&](int64_t j) {
+        const Item it = item(j);
+        uint64_t *bar = full + (j % stages);
+        unsigned char *st = data + (size_t)(j % stages) * stage_bytes;
+        const uint32_t bytes = it.ntok * H * row;
+        if (it.zero) {                      // nothing to fetch; the store side writes zeros itself
+            if (lane == 0) mbar_arrive(bar);
+            return;
+        }
+        if (lane == 0) mbar_arrive_expect(bar, bytes);
+        __syncwarp();
+        const char *src = p.src.base + it.s_base;
+        if (src_flat && dst_flat) {                     // one contiguous run on both sides
+            if (lane == 0) bulk_g2s(st, src, bytes, bar);
+        } else if (src_tok_major == dst_tok_major) {    // same order: one run per head (or per token)
+            const uint32_t outer = dst_tok_major ? it.ntok : H;
+            const uint32_t run = (dst_tok_major ? H : it.ntok) * row;
+            const int64_t s_outer = dst_tok_major ? p.src.tok_stride : p.src.head_stride;
+            const int64_t s_inner = dst_tok_major ? p.src.head_stride : p.src.tok_stride;
+            if (s_inner == (int64_t)row) {
+                for (uint32_t o = lane; o < outer; o += 32) bulk_g2s(st + (size_t)o * run, src + o * s_outer, run, bar);
+            } else {                                    // rows of a run are not adjacent in the source
+                const uint32_t inner = dst_tok_major ? H : it.ntok;
+                const uint32_t m_in = dst_tok_major ? m_H : div_magic(inner);
+                for (uint32_t r = lane; r < outer * inner; r += 32) {
+                    const uint32_t o = fast_div(r, m_in), i = r - o * inner;
+                    bulk_g2s(st + (size_t)r * row, src + o * s_outer + i * s_inner, row, bar);
+                }
+            }
+        } else {                                        // transpose: one bulk copy per row
+            const uint32_t inner = dst_tok_major ? H : it.ntok;   // inner index of the stage layout
+            const uint32_t m_in = dst_tok_major ? m_H : div_magic(inner);
+            const uint32_t rows = it.ntok * H;
+            for (uint32_t r = lane; r < rows; r += 32) {
+                const uint32_t o = fast_div(r, m_in), i = r - o * inner;
+                const uint32_t tk = dst_tok_major ? o : i, hd = dst_tok_major ? i : o;
+                bulk_g2s(st + (size_t)r * row, src + tk * p.src.tok_stride + hd * p.src.head_stride, row, bar);
+            }
+        }
+    };
+
+    // Write item j from its stage (or zeros) to the destination.
+    auto issue_store = [&](int64_t j) {
+        const Item it = item(j);
+        unsigned char *st = data + (size_t)(j % stages) * stage_bytes;
+        char *dst = p.dst.base + it.d_base;
+        if (it.zero) {                      // tail slots: plain 16-byte stores of zeros
+            const uint32_t vpr = row / 16;
+            const uint32_t outer = dst_tok_major ? it.ntok : H, inner = dst_tok_major ? H : it.ntok;
+            const int64_t d_outer = dst_tok_major ? p.dst.tok_stride : p.dst.head_stride;
+            const int64_t d_inner = dst_tok_major ? p.dst.head_stride : p.dst.tok_stride;
+            const uint32_t m_vpr = div_magic(vpr), m_in = div_magic(inner);
+            const uint32_t nvec = outer * inner * vpr;
+            for (uint32_t v = lane; v < nvec; v += 32) {
+                const uint32_t r = fast_div(v, m_vpr), vv = v - r * vpr;
+                const uint32_t o = fast_div(r, m_in), i = r - o * inner;
+                __stcs(reinterpret_cast<uint4 *>(dst + o * d_outer + i * d_inner + (int64_t)vv * 16),
+                       make_uint4(0, 0, 0, 0));
+            }
+            return;
+        }
+        if (dst_flat) {
+            if (lane == 0) bulk_s2g(dst, st, it.ntok * H * row);
+        } else if (dst_tok_major) {         // token-major with gaps between tokens cannot occur for our sides,
+            for (uint32_t tk = lane; tk < it.ntok; tk += 32)   // but keep it correct: one run per token
+                bulk_s2g(dst + tk * p.dst.tok_stride, st + (size_t)tk * H * row, H * row);
+        } else {                            // head-major: one run per head
+            const uint32_t run = it.ntok * row;
+            for (uint32_t hd = lane; hd < H; hd += 32) bulk_s2g(dst + hd * p.dst.head_stride, st + (size_t)hd * run, run);
+        }
+        bulk_commit();
+    };
+
+    int64_t head = 0;
+    for (int64_t tail = 0; tail < n_mine; ++tail) {
+        while (head < n_mine && head < tail + stages) {
+            if (head >= stages) {           // the stage was read by an earlier store of this warp
+                bulk_wait_read_all();
+                __syncwarp();
+            }
+            issue_load(head);
+            ++head;
+        }
+        uint64_t *bar = full + (tail % stages);
+        const uint32_t phase = (uint32_t)((tail / stages) & 1);
+        uint32_t spins = 0;
+        bool ok = true;
+        while (!mbar_try_wait(bar, phase)) {
+            if (++spins > kSpinLimit) {
+                ok = false;
+                break;
+            }
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) {                           // give up: record where, drain our stores, leave
+            if (lane == 0 && atomicCAS(p.status, 0ull, 2ull) == 0ull) p.status[1] = (unsigned long long)tail;
+            bulk_wait_all();
+            for (int64_t j = tail + 1; j < head; ++j) {   // loads still aimed at our stages: bounded wait each
+                uint32_t s2 = 0;
+                while (!mbar_try_wait(full + (j % stages), (uint32_t)((j / stages) & 1)) && ++s2 <= kSpinLimit) {}
+            }
+            return;
+        }
+        issue_store(tail);
+    }
+    bulk_wait_all();
+}
+
+cudaError_t launch_bulk(const CopyParams &p, const LaunchConfig &cfg, cudaStream_t stream)
+{
+    const int64_t n_work = (int64_t)p.n_tiles * p.n_lc;
+    if (n_work <= 0) return cudaSuccess;
+    const uint32_t stage_bytes = (uint32_t)((cfg.max_tile_bytes + 127) / 128 * 128);
+    const int stages = cfg.stages;
+    const size_t smem = kBarrierBytes + (size_t)stages * stage_bytes;
+    cudaError_t e = cudaFuncSetAttribute(bulk_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int occ = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, bulk_tiles_kernel, 32, smem);
+    if (e != cudaSuccess) return e;
+    if (occ < 1) return cudaErrorInvalidConfiguration;
+    if (occ > cfg.ctas_per_sm) occ = cfg.ctas_per_sm;
+    int64_t grid = (int64_t)cfg.sm_count * occ;
+    if (grid > n_work) grid = n_work;
+    bulk_tiles_kernel<<<(unsigned)grid, 32, smem, stream>>>(p, stages, stage_bytes);
+    return cudaGetLastError();
+}
+
+// The bulk path needs 16-byte rows and a tile that fits a stage (and the
+// mbarrier's transaction counter); otherwise the register path is used.
+bool bulk_supported(const LaunchConfig &cfg, int row_bytes)
+{
+    const size_t smem = kBarrierBytes + (size_t)cfg.stages * ((cfg.max_tile_bytes + 127) / 128 * 128);
+    return row_bytes % 16 == 0 && cfg.vec_bytes >= 16 && cfg.max_tile_bytes > 0 && cfg.max_tile_bytes <= 131072 &&
+           smem <= 220 * 1024 && cfg.stages >= 2 && !cfg.check_bounds;
+}
+
+}  // namespace pdkv

@@ -49,11 +49,17 @@ struct LaunchConfig {
     int ctas_per_sm;
     int sm_count;
     int variant;
+    int stages;              // bulk variant: shared-memory stages per CTA
+    int64_t max_tile_bytes;  // bulk variant: largest tile of the launch
     bool check_bounds;
 };
 
 // Enqueue one persistent copy kernel.  Returns the CUDA status of the launch.
 cudaError_t launch_copy(const CopyParams &p, const LaunchConfig &cfg, cudaStream_t stream);
+
+// Bulk-copy (TMA) variant: same contract; bulk_supported() says whether a launch qualifies.
+cudaError_t launch_bulk(const CopyParams &p, const LaunchConfig &cfg, cudaStream_t stream);
+bool bulk_supported(const LaunchConfig &cfg, int row_bytes);
 
 struct Tunables {
     int64_t tile_bytes = 65536;
@@ -65,6 +71,7 @@ struct Tunables {
     int64_t chunked = 0;
     int64_t debug_bounds = 0;
     int64_t variant = 0;
+    int64_t stages = 3;
     int64_t dry_run = 0;
 };
 Tunables &tunables();

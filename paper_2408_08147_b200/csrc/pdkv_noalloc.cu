@@ -114,6 +114,8 @@ extern "C" int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
         cfg.ctas_per_sm = (int)t.ctas_per_sm;
         cfg.sm_count = slot.sm_count;
         cfg.variant = 0;
+        cfg.stages = 0;
+        cfg.max_tile_bytes = 0;
         cfg.check_bounds = false;
         if ((e = pdkv::launch_copy(p, cfg, st)) != cudaSuccess) rc = pdkv::report_cuda_error(e, "kernel launch");
     }

@@ -25,6 +25,8 @@ def _gpu_lib():
     B.pdkv_tune("debug_bounds", 0)
     B.pdkv_tune("tile_bytes", 65536)
     B.pdkv_tune("lc_fastest", 0)
+    B.pdkv_tune("variant", 0)
+    B.pdkv_tune("stages", 3)
 
 
 def dev(a: np.ndarray):
@@ -120,6 +122,35 @@ def test_tile_size_and_work_order_do_not_change_the_result(oracle, tile_bytes, l
     finally:
         B.pdkv_tune("tile_bytes", 65536)
         B.pdkv_tune("lc_fastest", 0)
+
+
+@pytest.mark.parametrize("stages,tile_bytes,chunked", [(2, 16384, 0), (3, 65536, 0), (4, 32768, 1)])
+def test_bulk_copy_variant(oracle, stages, tile_bytes, chunked):
+    """Variant 1 (TMA bulk copies through a shared-memory ring) must produce the
+    same bytes: flat, head-run and transposing tiles, zero-fill tiles, skip masks."""
+    B.pdkv_tune("variant", 1)
+    B.pdkv_tune("stages", stages)
+    B.pdkv_tune("tile_bytes", tile_bytes)
+    B.pdkv_tune("chunked", chunked)
+    try:
+        check_all_ops(oracle, W.make_config(1))
+        check_all_ops(oracle, W.make_config(2, num_layers=2, n_req=5, max_len=640))
+        check_all_ops(oracle, W.make_config(2, num_layers=2, n_req=4, max_len=600, src_layout=W.LAYER_MAJOR))
+        check_all_ops(oracle, W.make_config(3, num_layers=2, n_req=10, max_len=1500), side_stream=True)
+        check_all_ops(oracle, W.make_config(5, num_layers=2, n_req=30), layers=(1, 2))
+        check_all_ops(oracle, W.make_config(3, num_layers=2, n_req=6, max_len=900, src_layout=W.LAYER_MAJOR,
+                                            dst_layout=W.BLOCK_MAJOR))
+        # odd block sizes and head counts, 16-byte rows
+        lens = np.array([0, 37, 5, 90], np.int32)
+        w = W.build_workload("odd", 7, num_layers=2, num_kv_heads=3, head_dim=8, elem_bytes=2, seq_len=lens,
+                             src_layout=W.BLOCK_MAJOR, src_block=7, dst_layout=W.LAYER_MAJOR, dst_block=5,
+                             src_slack=1.3, dst_slack=1.3)
+        check_all_ops(oracle, w)
+    finally:
+        B.pdkv_tune("variant", 0)
+        B.pdkv_tune("stages", 3)
+        B.pdkv_tune("tile_bytes", 65536)
+        B.pdkv_tune("chunked", 0)
 
 
 @pytest.mark.parametrize("seed", range(16))
