@@ -517,6 +517,91 @@ def e2e_leg(args, w, src_t, dst_t, buf_t, stream, step_bytes, torch, B, Transfer
                         "D2H decode pool to pinned memory"}
 
 
+def overlap_arm(args):
+    """Per-layer trigger (Sec. 3.5): layer l is transferred on a side stream as soon
+    as a stand-in for layer l's compute (one bf16 GEMM on the main stream) has
+    finished, while layer l+1 computes.  Reports compute alone, transfer alone,
+    and both overlapped, for the register and the bulk-copy variants."""
+    import torch
+
+    from paper_2408_08147_b200 import binding as B
+    from paper_2408_08147_b200 import workloads as W
+    from paper_2408_08147_b200.session import TransferSession
+
+    B.lib()
+    torch.cuda.set_device(0)
+    kw = {"n_req": args.n_req} if args.n_req else {}
+    w = W.make_config(args.config, **kw)
+    src_t, dst_t = alloc_pools(w, torch)
+    L = w.src.num_layers
+    n = args.gemm_n
+    a = torch.randn(n, n, device="cuda", dtype=torch.bfloat16)
+    b = torch.randn(n, n, device="cuda", dtype=torch.bfloat16)
+    c = torch.empty(n, n, device="cuda", dtype=torch.bfloat16)
+    # the transfer stream gets the higher priority: its CTAs are placed as soon as
+    # a compute CTA retires instead of after the whole compute grid
+    main, side = torch.cuda.Stream(), torch.cuda.Stream(priority=-1 if args.side_priority else 0)
+    torch.cuda.synchronize()
+
+    def timed(fn, reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        fn()
+        torch.cuda.synchronize()
+        e0.record(main)
+        for _ in range(reps):
+            fn()
+        side_done = torch.cuda.Event()
+        side_done.record(side)
+        main.wait_event(side_done)
+        e1.record(main)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    def compute_only():
+        with torch.cuda.stream(main):
+            for _ in range(L):
+                torch.matmul(a, b, out=c)
+
+    results = {}
+    modes = [("register copy, defaults", {"variant": 0}),
+             ("register copy, 1 CTA/SM", {"variant": 0, "ctas_per_sm": 1, "threads": 512, "unroll": 2}),
+             ("bulk copy (TMA), 8 KiB tiles x 2 stages x 8 CTAs/SM",
+              {"variant": 1, "tile_bytes": 8192, "stages": 2, "ctas_per_sm": 8})]
+    defaults = {k: B.pdkv_tune_get(k) for k in ("variant", "ctas_per_sm", "threads", "unroll", "tile_bytes", "stages")}
+    t_compute = timed(compute_only, args.steps)
+    for name, tune in modes:
+        for k, v in {**defaults, **tune}.items():
+            B.pdkv_tune(k, v)
+        sess = TransferSession(w.src, src_t, w.dst, dst_t, w.batch, side.cuda_stream)
+
+        def transfer_only():
+            for l in range(L):
+                sess.transfer((l, l + 1), side.cuda_stream)
+
+        def overlapped():
+            for l in range(L):
+                with torch.cuda.stream(main):
+                    torch.matmul(a, b, out=c)
+                    ev = torch.cuda.Event()
+                    ev.record(main)
+                side.wait_event(ev)
+                sess.transfer((l, l + 1), side.cuda_stream)
+
+        t_x = timed(transfer_only, args.steps)
+        t_o = timed(overlapped, args.steps)
+        results[name] = {"transfer_alone_ms": t_x, "overlapped_ms": t_o,
+                         "serial_ms": t_compute + t_x,
+                         "hidden_fraction_of_transfer": max(0.0, min(1.0, (t_compute + t_x - t_o) / t_x))}
+        sess.close()
+    for k, v in defaults.items():
+        B.pdkv_tune(k, v)
+    out = {"mode": "overlap", "config": {"workload": workload_name(w), "layers": L,
+                                         "compute_stand_in": f"{L} x torch.matmul bf16 {n}^3 on the main stream",
+                                         "transfer_stream_priority": "high" if args.side_priority else "default"},
+           "compute_alone_ms": t_compute, "variants": results}
+    print(json.dumps(out), flush=True)
+
+
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -533,6 +618,9 @@ def parse():
     ap.add_argument("--no-extras", action="store_true", help="skip baseline, e2e and CPU legs")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--overlap", action="store_true", help="per-layer transfer overlapped with a compute stand-in")
+    ap.add_argument("--gemm-n", type=int, default=4096)
+    ap.add_argument("--side-priority", type=int, default=1, help="1: transfer stream has high priority")
     ap.add_argument("--no-blockwise", action="store_true")
     return ap.parse_args()
 
@@ -540,7 +628,9 @@ def parse():
 if __name__ == "__main__":
     a = parse()
     a.warmup = max(a.warmup, 3) if a.impl == "pdkv" else a.warmup
-    if a.impl == "reference":
+    if a.overlap:
+        overlap_arm(a)
+    elif a.impl == "reference":
         reference_arm(a)
     else:
         main_arm(a)
