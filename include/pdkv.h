@@ -210,6 +210,23 @@ int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
  * Same result as pdkv_transfer over all layers. */
 int pdkv_transfer_blockwise(const pdkv_plan *plan, void *stream);
 
+/* Host-resident pools.  `host_src_pool` / `host_dst_pool` (host; pinned memory
+ * makes the copies asynchronous) are byte images of the prefill / decode pool
+ * with the pool's own geometry.  pdkv_upload_blocks() copies every prefill
+ * block that holds at least one kept token of the batch into the device pool
+ * at the same offsets; pdkv_download_blocks() copies every decode block the
+ * batch writes back out.  Consecutive block ids travel as one (pitched) copy;
+ * other bytes of either image are not touched.  Both only enqueue on
+ * `stream`.  With pack / unpack / transfer in between, this is the whole path
+ * for a caller whose KV lives in host memory.  (No counterpart in Sec. 3.5,
+ * which moves device to device; the paper's discussion section mentions a
+ * host-memory KV pool as orthogonal work.)
+ * pdkv_plan_block_bytes() reports the bytes each of the two calls moves.
+ * Errors: INVALID_ARG, CUDA. */
+int pdkv_upload_blocks(const pdkv_plan *plan, const void *host_src_pool, void *stream);
+int pdkv_download_blocks(const pdkv_plan *plan, void *host_dst_pool, void *stream);
+int pdkv_plan_block_bytes(const pdkv_plan *plan, uint64_t *src_bytes, uint64_t *dst_bytes);
+
 /* Number of GPU operations (kernel launches + memcpys) one call of `op`
  * enqueues; op = 3 asks about pdkv_transfer_blockwise. */
 int pdkv_plan_launches(const pdkv_plan *plan, int op, int64_t *launches);

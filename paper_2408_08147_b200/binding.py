@@ -39,7 +39,7 @@ EXPORTS = (
     "pdkv_pool_bytes", "pdkv_pool_create", "pdkv_pool_destroy", "pdkv_plan_create",
     "pdkv_plan_destroy", "pdkv_plan_buffer", "pdkv_plan_traffic", "pdkv_pack", "pdkv_unpack",
     "pdkv_transfer", "pdkv_transfer_noalloc", "pdkv_transfer_blockwise", "pdkv_plan_launches", "pdkv_plan_tiles",
-    "pdkv_plan_status", "pdkv_tune", "pdkv_tune_get", "pdkv_strerror",
+    "pdkv_plan_status", "pdkv_upload_blocks", "pdkv_download_blocks", "pdkv_plan_block_bytes", "pdkv_tune", "pdkv_tune_get", "pdkv_strerror",
 )
 
 
@@ -99,6 +99,9 @@ def lib() -> C.CDLL:
     L.pdkv_plan_launches.argtypes = [vp, C.c_int, C.POINTER(i64)]
     L.pdkv_plan_tiles.argtypes = [vp, C.c_int, C.POINTER(C.POINTER(pdkv_tile)), C.POINTER(i64)]
     L.pdkv_plan_status.argtypes = [vp, vp]
+    L.pdkv_upload_blocks.argtypes = [vp, vp, vp]
+    L.pdkv_download_blocks.argtypes = [vp, vp, vp]
+    L.pdkv_plan_block_bytes.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     L.pdkv_tune.argtypes = [C.c_char_p, i64]
     L.pdkv_tune_get.argtypes = [C.c_char_p, C.POINTER(i64)]
     L.pdkv_strerror.restype = C.c_char_p
@@ -247,6 +250,23 @@ def pdkv_plan_tiles(plan: int, op: int) -> np.ndarray:
 
 def pdkv_plan_status(plan: int, stream: int = 0) -> None:
     _check(lib().pdkv_plan_status(C.c_void_p(plan), C.c_void_p(stream)), "pdkv_plan_status")
+
+
+def pdkv_upload_blocks(plan: int, host_src_ptr: int, stream: int = 0) -> None:
+    _check(lib().pdkv_upload_blocks(C.c_void_p(plan), C.c_void_p(host_src_ptr), C.c_void_p(stream)),
+           "pdkv_upload_blocks")
+
+
+def pdkv_download_blocks(plan: int, host_dst_ptr: int, stream: int = 0) -> None:
+    _check(lib().pdkv_download_blocks(C.c_void_p(plan), C.c_void_p(host_dst_ptr), C.c_void_p(stream)),
+           "pdkv_download_blocks")
+
+
+def pdkv_plan_block_bytes(plan: int):
+    """(bytes pdkv_upload_blocks copies, bytes pdkv_download_blocks copies)."""
+    a, b = C.c_uint64(), C.c_uint64()
+    _check(lib().pdkv_plan_block_bytes(C.c_void_p(plan), C.byref(a), C.byref(b)), "pdkv_plan_block_bytes")
+    return int(a.value), int(b.value)
 
 
 def pdkv_tune(key: str, value: int) -> None:

@@ -88,6 +88,8 @@ struct pdkv_plan {
     std::vector<Tile> tiles[3];
     const Tile *dev_tiles[3] = {nullptr, nullptr, nullptr};
     std::vector<BlockGroup> groups;
+    // maximal runs of consecutive block ids: prefill blocks the batch reads, decode blocks it writes
+    std::vector<std::pair<int64_t, int64_t>> src_runs, dst_runs;  // (first id, count)
     void *dev_mem = nullptr;
     unsigned long long *dev_status = nullptr;
     int vec_bytes = 16;
@@ -401,6 +403,32 @@ int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip_gr
                 if (batch->dst_tbl_off[r + 1] - batch->dst_tbl_off[r] < need) return PDKV_ERR_TABLE;
             }
         }
+        auto runs_of = [](const std::vector<uint8_t> &seen, std::vector<std::pair<int64_t, int64_t>> &out) {
+            for (size_t i = 0; i < seen.size();) {
+                if (!seen[i]) {
+                    ++i;
+                    continue;
+                }
+                size_t j = i;
+                while (j < seen.size() && seen[j]) ++j;
+                out.emplace_back((int64_t)i, (int64_t)(j - i));
+                i = j;
+            }
+        };
+        if (src) {  // prefill blocks holding at least one kept token
+            std::vector<uint8_t> seen((size_t)src->d.num_blocks, 0);
+            const int64_t Bp = src->d.block_tokens;
+            for (int32_t r = 0; r < batch->n_req; ++r) {
+                const int64_t len = batch->seq_len[r];
+                const uint8_t *skip = batch->dst_skip ? batch->dst_skip + batch->dst_tbl_off[r] : nullptr;
+                for (int64_t t = 0; t < len;) {
+                    const int64_t next = std::min(len, std::min((t / Bp + 1) * Bp, (t / G + 1) * (int64_t)G));
+                    if (!(skip && skip[t / G])) seen[(size_t)batch->src_tbl[batch->src_tbl_off[r] + t / Bp]] = 1;
+                    t = next;
+                }
+            }
+            runs_of(seen, pl->src_runs);
+        }
         if (dst) {  // every written decode block has exactly one writer
             std::vector<uint8_t> seen((size_t)dst->d.num_blocks, 0);
             const int64_t Bd = dst->d.block_tokens;
@@ -414,6 +442,7 @@ int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip_gr
                     s = 1;
                 }
             }
+            runs_of(seen, pl->dst_runs);
         }
 
         // kept tokens and buffer offsets
@@ -606,6 +635,70 @@ int pdkv_transfer_blockwise(const pdkv_plan *plan, void *stream)
             if (rc != PDKV_OK) return rc;
         }
     }
+    return PDKV_OK;
+}
+
+namespace {
+
+// Copy whole blocks between a host image of a pool and the device pool, one
+// (strided) copy per run of consecutive block ids.
+int copy_block_runs(const pdkv_pool &pool, const std::vector<std::pair<int64_t, int64_t>> &runs,
+                    char *host_base, bool to_device, int64_t row, int64_t hrow, cudaStream_t st)
+{
+    const pdkv_pool_desc &d = pool.d;
+    const cudaMemcpyKind kind = to_device ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost;
+    for (const auto &run : runs) {
+        cudaError_t e;
+        if (d.layout == PDKV_LAYOUT_BLOCK_MAJOR) {
+            const size_t blk = (size_t)2 * d.num_layers * d.block_tokens * hrow;
+            char *dev = pool.base + (size_t)run.first * blk, *host = host_base + (size_t)run.first * blk;
+            e = cudaMemcpyAsync(to_device ? dev : host, to_device ? host : dev, (size_t)run.second * blk, kind, st);
+        } else {  // [layer][K/V][block]...: 2*L pieces per run, one pitched copy
+            const size_t blk = (size_t)d.num_kv_heads * d.block_tokens * row;
+            const size_t pitch = (size_t)d.num_blocks * blk;
+            char *dev = pool.base + (size_t)run.first * blk, *host = host_base + (size_t)run.first * blk;
+            e = cudaMemcpy2DAsync(to_device ? dev : host, pitch, to_device ? host : dev, pitch,
+                                  (size_t)run.second * blk, (size_t)2 * d.num_layers, kind, st);
+        }
+        if (e != cudaSuccess) return cuda_fail(e, to_device ? "host-to-device block copy" : "device-to-host block copy");
+    }
+    return PDKV_OK;
+}
+
+}  // namespace
+
+int pdkv_upload_blocks(const pdkv_plan *plan, const void *host_src_pool, void *stream)
+{
+    if (!plan || !plan->has_src || !plan->dev_mem) return PDKV_ERR_INVALID_ARG;
+    if (plan->src_runs.empty()) return PDKV_OK;
+    if (!host_src_pool) return PDKV_ERR_INVALID_ARG;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    return copy_block_runs(plan->src, plan->src_runs, const_cast<char *>(static_cast<const char *>(host_src_pool)),
+                           true, plan->row_bytes, plan->hrow_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int pdkv_download_blocks(const pdkv_plan *plan, void *host_dst_pool, void *stream)
+{
+    if (!plan || !plan->has_dst || !plan->dev_mem) return PDKV_ERR_INVALID_ARG;
+    if (plan->dst_runs.empty()) return PDKV_OK;
+    if (!host_dst_pool) return PDKV_ERR_INVALID_ARG;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    return copy_block_runs(plan->dst, plan->dst_runs, static_cast<char *>(host_dst_pool), false, plan->row_bytes,
+                           plan->hrow_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int pdkv_plan_block_bytes(const pdkv_plan *plan, uint64_t *src_bytes, uint64_t *dst_bytes)
+{
+    if (!plan) return PDKV_ERR_INVALID_ARG;
+    auto total = [&](const pdkv_pool &pool, const std::vector<std::pair<int64_t, int64_t>> &runs) {
+        uint64_t n = 0;
+        for (const auto &r : runs) n += (uint64_t)r.second;
+        return n * 2ull * pool.d.num_layers * pool.d.block_tokens * (uint64_t)plan->hrow_bytes;
+    };
+    if (src_bytes) *src_bytes = plan->has_src ? total(plan->src, plan->src_runs) : 0;
+    if (dst_bytes) *dst_bytes = plan->has_dst ? total(plan->dst, plan->dst_runs) : 0;
     return PDKV_OK;
 }
 

@@ -68,6 +68,17 @@ class TransferSession:
     def transfer_blockwise(self, stream: Optional[int] = None) -> None:
         B.pdkv_transfer_blockwise(self.plan, self.stream if stream is None else stream)
 
+    def upload_blocks(self, host_src_t, stream: Optional[int] = None) -> None:
+        """H2D of the prefill blocks the batch reads, from a host image of the pool."""
+        B.pdkv_upload_blocks(self.plan, host_src_t.data_ptr(), self.stream if stream is None else stream)
+
+    def download_blocks(self, host_dst_t, stream: Optional[int] = None) -> None:
+        """D2H of the decode blocks the batch writes, into a host image of the pool."""
+        B.pdkv_download_blocks(self.plan, host_dst_t.data_ptr(), self.stream if stream is None else stream)
+
+    def block_bytes(self):
+        return B.pdkv_plan_block_bytes(self.plan)
+
     def status(self, stream: Optional[int] = None) -> None:
         B.pdkv_plan_status(self.plan, self.stream if stream is None else stream)
 

@@ -241,3 +241,43 @@ def test_per_layer_calls_equal_whole_model(oracle):
             s.transfer((l, l + 1))
         s.status()
         assert np.array_equal(host(dst_t), want)
+
+
+@pytest.mark.parametrize("idx,kw", [(5, dict(num_layers=2, n_req=30, src_block=32)),
+                                    (3, dict(num_layers=2, n_req=6, max_len=700, src_layout=W.LAYER_MAJOR,
+                                             dst_layout=W.BLOCK_MAJOR)),
+                                    (4, dict(num_layers=2, n_req=3, max_len=500))])
+def test_host_resident_pools(oracle, idx, kw):
+    """Upload the referenced prefill blocks from a host image, transfer, download
+    the written decode blocks: the host decode image must equal the checker's,
+    and nothing else may move in either direction."""
+    from paper_2408_08147_b200.session import TransferSession
+
+    w = W.make_config(idx, **kw)
+    src = W.fill_pool_numpy(w.src, w.seed)
+    sent = W.sentinel_pool_numpy(w.dst)
+    want = sent.copy()
+    oracle.transfer(w.src, src, w.dst, want, w.batch)
+    h_src = torch.from_numpy(src.view(np.uint8).copy()).pin_memory()
+    h_dst = torch.from_numpy(sent.view(np.uint8).copy()).pin_memory()
+    src_t = torch.full((w.src.num_bytes(),), 0x5A, dtype=torch.uint8, device="cuda")
+    dst_t = dev(sent)
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with TransferSession(w.src, src_t, w.dst, dst_t, w.batch, stream.cuda_stream) as s:
+        up, down = s.block_bytes()
+        s.upload_blocks(h_src)
+        s.transfer()
+        s.download_blocks(h_dst)
+        s.status()
+    assert np.array_equal(h_dst.numpy().view(np.uint16), want)
+    # device prefill pool: uploaded blocks equal the host image, all others keep the 0x5A fill
+    got_src = src_t.cpu().numpy()
+    same = got_src == src.view(np.uint8)
+    untouched = got_src == 0x5A
+    assert (same | untouched).all()
+    not_uploaded = w.src.num_bytes() - up          # bytes of blocks the batch does not read
+    assert not_uploaded * 0.98 <= int((~same).sum()) <= not_uploaded   # (1/256 of the fill matches by chance)
+    assert up <= w.src.num_bytes() and down <= w.dst.num_bytes()
+    if w.src_occupied.size or w.batch.dst_skip is not None:
+        assert up < w.src.num_bytes()

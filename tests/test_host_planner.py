@@ -265,3 +265,24 @@ def test_tiles_respect_size_cap_and_block_boundaries():
     assert B.pdkv_plan_launches(plan, B.PDKV_OP_TRANSFER) == 1
     B.pdkv_plan_destroy(plan)
     B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
+
+
+def test_block_bytes_count_referenced_and_written_blocks():
+    w = W.make_config(5, num_layers=2, n_req=60, src_block=32)
+    ps, pd = _pools(w)
+    plan = _plan(w, ps, pd)
+    b = w.batch
+    src_ids, dst_ids = set(), set()
+    for r in range(b.n_req):
+        for t in range(int(b.seq_len[r])):
+            e = b.dst_tbl_off[r] + t // w.dst.block_tokens
+            if b.dst_skip[e]:
+                continue
+            dst_ids.add(int(b.dst_tbl[e]))
+            src_ids.add(int(b.src_tbl[b.src_tbl_off[r] + t // w.src.block_tokens]))
+    blk_src = w.src.num_bytes() // w.src.num_blocks
+    blk_dst = w.dst.num_bytes() // w.dst.num_blocks
+    assert B.pdkv_plan_block_bytes(plan) == (len(src_ids) * blk_src, len(dst_ids) * blk_dst)
+    assert len(src_ids) < w.src.num_blocks            # resident prefixes are not uploaded
+    B.pdkv_plan_destroy(plan)
+    B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
