@@ -59,6 +59,7 @@ extern "C" {
 
 typedef struct pdkv_pool pdkv_pool; /* opaque: geometry + borrowed device base */
 typedef struct pdkv_plan pdkv_plan; /* opaque: validated batch + device tile lists */
+typedef struct pdkv_queue pdkv_queue; /* opaque: receive slots for asynchronous retrieval */
 
 enum pdkv_layout {
     PDKV_LAYOUT_BLOCK_MAJOR = 0,
@@ -74,7 +75,8 @@ enum pdkv_status {
     PDKV_ERR_CUDA = -5,             /* a CUDA runtime call failed */
     PDKV_ERR_DEVICE_BOUNDS = -6,    /* bounds-checked kernels refused an access (debug option) */
     PDKV_ERR_NOMEM = -7,            /* host allocation failed */
-    PDKV_ERR_LIMIT = -8             /* batch larger than pdkv_transfer_noalloc's built-in scratch */
+    PDKV_ERR_LIMIT = -8,            /* batch larger than pdkv_transfer_noalloc's built-in scratch */
+    PDKV_ERR_BUSY = -9              /* pdkv_queue_submit: every receive slot is taken */
 };
 
 enum pdkv_op {
@@ -226,6 +228,43 @@ int pdkv_transfer_blockwise(const pdkv_plan *plan, void *stream);
 int pdkv_upload_blocks(const pdkv_plan *plan, const void *host_src_pool, void *stream);
 int pdkv_download_blocks(const pdkv_plan *plan, void *host_dst_pool, void *stream);
 int pdkv_plan_block_bytes(const pdkv_plan *plan, uint64_t *src_bytes, uint64_t *dst_bytes);
+
+/* Asynchronous retrieval, Sec. 3.5: the decode side has little room for
+ * incoming KVCache, so the space forms a small queue of `capacity` (1..64)
+ * receive slots; retrieval runs concurrently with decoding and a completed
+ * request triggers the next retrieval, on demand.
+ *
+ *   pdkv_queue_create   one non-blocking stream and one event per slot on
+ *                       `device`; the pools are borrowed until destroy.
+ *   pdkv_queue_submit   takes a free slot, builds the plan for `batch` (host
+ *                       arrays, read during the call) and enqueues the fused
+ *                       transfer over all layers on the slot's stream --
+ *                       preceded by pdkv_upload_blocks() if `host_src_pool` is
+ *                       given and followed by pdkv_download_blocks() if
+ *                       `host_dst_pool` is given (either may be NULL).  Returns a
+ *                       ticket.  If every slot is taken it returns PDKV_ERR_BUSY at
+ *                       once and enqueues nothing: nothing waits inside the library,
+ *                       the caller retries when a request completes.
+ *   pdkv_queue_poll     *done = 1 once the slot's transfer has finished (its
+ *                       decode blocks are valid for the next decode iteration).
+ *   pdkv_queue_wait     blocks the calling thread until then.
+ *   pdkv_queue_release  hands the slot back (waits for the transfer if it is
+ *                       still running); the ticket becomes invalid.
+ *   pdkv_queue_stats    capacity, slots in use, accepted and rejected submits.
+ * Concurrent tickets must write disjoint decode blocks (the caller's block
+ * allocator guarantees that).  Calls on one queue are serialised by a mutex.
+ * Errors: INVALID_ARG (unknown ticket, bad arguments), BUSY, and whatever
+ * pdkv_plan_create / pdkv_transfer return. */
+int pdkv_queue_create(const pdkv_pool *src, const pdkv_pool *dst, int device, int capacity,
+                      pdkv_queue **out);
+int pdkv_queue_submit(pdkv_queue *queue, const pdkv_batch_desc *batch, const void *host_src_pool,
+                      void *host_dst_pool, int64_t *ticket);
+int pdkv_queue_poll(pdkv_queue *queue, int64_t ticket, int *done);
+int pdkv_queue_wait(pdkv_queue *queue, int64_t ticket);
+int pdkv_queue_release(pdkv_queue *queue, int64_t ticket);
+int pdkv_queue_stats(const pdkv_queue *queue, int *capacity, int *in_use, int64_t *submitted,
+                     int64_t *rejected);
+int pdkv_queue_destroy(pdkv_queue *queue);
 
 /* Number of GPU operations (kernel launches + memcpys) one call of `op`
  * enqueues; op = 3 asks about pdkv_transfer_blockwise. */

@@ -28,6 +28,7 @@ PDKV_ERR_CUDA = -5
 PDKV_ERR_DEVICE_BOUNDS = -6
 PDKV_ERR_NOMEM = -7
 PDKV_ERR_LIMIT = -8
+PDKV_ERR_BUSY = -9
 PDKV_NOALLOC_MAX_TILES = 32768
 
 PDKV_OP_PACK = 0
@@ -39,7 +40,9 @@ EXPORTS = (
     "pdkv_pool_bytes", "pdkv_pool_create", "pdkv_pool_destroy", "pdkv_plan_create",
     "pdkv_plan_destroy", "pdkv_plan_buffer", "pdkv_plan_traffic", "pdkv_pack", "pdkv_unpack",
     "pdkv_transfer", "pdkv_transfer_noalloc", "pdkv_transfer_blockwise", "pdkv_plan_launches", "pdkv_plan_tiles",
-    "pdkv_plan_status", "pdkv_upload_blocks", "pdkv_download_blocks", "pdkv_plan_block_bytes", "pdkv_tune", "pdkv_tune_get", "pdkv_strerror",
+    "pdkv_plan_status", "pdkv_upload_blocks", "pdkv_download_blocks", "pdkv_plan_block_bytes",
+    "pdkv_queue_create", "pdkv_queue_submit", "pdkv_queue_poll", "pdkv_queue_wait", "pdkv_queue_release",
+    "pdkv_queue_stats", "pdkv_queue_destroy", "pdkv_tune", "pdkv_tune_get", "pdkv_strerror",
 )
 
 
@@ -102,6 +105,13 @@ def lib() -> C.CDLL:
     L.pdkv_upload_blocks.argtypes = [vp, vp, vp]
     L.pdkv_download_blocks.argtypes = [vp, vp, vp]
     L.pdkv_plan_block_bytes.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+    L.pdkv_queue_create.argtypes = [vp, vp, C.c_int, C.c_int, C.POINTER(vp)]
+    L.pdkv_queue_submit.argtypes = [vp, C.POINTER(pdkv_batch_desc), vp, vp, C.POINTER(i64)]
+    L.pdkv_queue_poll.argtypes = [vp, i64, C.POINTER(C.c_int)]
+    L.pdkv_queue_wait.argtypes = [vp, i64]
+    L.pdkv_queue_release.argtypes = [vp, i64]
+    L.pdkv_queue_stats.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(i64), C.POINTER(i64)]
+    L.pdkv_queue_destroy.argtypes = [vp]
     L.pdkv_tune.argtypes = [C.c_char_p, i64]
     L.pdkv_tune_get.argtypes = [C.c_char_p, C.POINTER(i64)]
     L.pdkv_strerror.restype = C.c_char_p
@@ -267,6 +277,52 @@ def pdkv_plan_block_bytes(plan: int):
     a, b = C.c_uint64(), C.c_uint64()
     _check(lib().pdkv_plan_block_bytes(C.c_void_p(plan), C.byref(a), C.byref(b)), "pdkv_plan_block_bytes")
     return int(a.value), int(b.value)
+
+
+def pdkv_queue_create(src_pool: int, dst_pool: int, device: int, capacity: int) -> int:
+    out = C.c_void_p()
+    _check(lib().pdkv_queue_create(C.c_void_p(src_pool), C.c_void_p(dst_pool), device, capacity,
+                                   C.byref(out)), "pdkv_queue_create")
+    return out.value
+
+
+def pdkv_queue_submit(queue: int, seq_len, src_tbl_off, src_tbl, dst_tbl_off, dst_tbl, dst_skip=None,
+                      host_src_ptr: Optional[int] = None, host_dst_ptr: Optional[int] = None):
+    """Returns a ticket, or ``None`` when every receive slot is taken."""
+    b = _BatchArrays(seq_len, src_tbl_off, src_tbl, dst_tbl_off, dst_tbl, dst_skip)
+    t = C.c_int64()
+    rc = lib().pdkv_queue_submit(C.c_void_p(queue), C.byref(b.desc), C.c_void_p(host_src_ptr),
+                                 C.c_void_p(host_dst_ptr), C.byref(t))
+    if rc == PDKV_ERR_BUSY:
+        return None
+    _check(rc, "pdkv_queue_submit")
+    return int(t.value)
+
+
+def pdkv_queue_poll(queue: int, ticket: int) -> bool:
+    d = C.c_int()
+    _check(lib().pdkv_queue_poll(C.c_void_p(queue), ticket, C.byref(d)), "pdkv_queue_poll")
+    return bool(d.value)
+
+
+def pdkv_queue_wait(queue: int, ticket: int) -> None:
+    _check(lib().pdkv_queue_wait(C.c_void_p(queue), ticket), "pdkv_queue_wait")
+
+
+def pdkv_queue_release(queue: int, ticket: int) -> None:
+    _check(lib().pdkv_queue_release(C.c_void_p(queue), ticket), "pdkv_queue_release")
+
+
+def pdkv_queue_stats(queue: int):
+    """(capacity, in_use, submitted, rejected)."""
+    cap, use, sub, rej = C.c_int(), C.c_int(), C.c_int64(), C.c_int64()
+    _check(lib().pdkv_queue_stats(C.c_void_p(queue), C.byref(cap), C.byref(use), C.byref(sub),
+                                  C.byref(rej)), "pdkv_queue_stats")
+    return cap.value, use.value, int(sub.value), int(rej.value)
+
+
+def pdkv_queue_destroy(queue: int) -> None:
+    _check(lib().pdkv_queue_destroy(C.c_void_p(queue)), "pdkv_queue_destroy")
 
 
 def pdkv_tune(key: str, value: int) -> None:

@@ -309,6 +309,8 @@ void describe_transfer(const pdkv_plan *plan, Side *src, Side *dst, int *H, int 
 
 int report_cuda_error(cudaError_t e, const char *what) { return cuda_fail(e, what); }
 
+int plan_num_layers(const pdkv_plan *plan) { return plan->L; }
+
 }  // namespace pdkv
 
 extern "C" {
@@ -794,6 +796,7 @@ const char *pdkv_strerror(int status)
     case PDKV_ERR_CUDA: return g_cuda_msg.empty() ? "CUDA error" : g_cuda_msg.c_str();
     case PDKV_ERR_DEVICE_BOUNDS: return g_cuda_msg.empty() ? "device bounds check refused an access" : g_cuda_msg.c_str();
     case PDKV_ERR_NOMEM: return "out of host memory";
+    case PDKV_ERR_BUSY: return "no free receive slot";
     case PDKV_ERR_LIMIT: return "batch exceeds the built-in scratch of the no-allocation entry point";
     default: return "unknown status";
     }

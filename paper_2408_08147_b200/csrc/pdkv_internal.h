@@ -83,5 +83,6 @@ int create_host_plan(const pdkv_pool *src, const pdkv_pool *dst, const pdkv_batc
 void describe_transfer(const pdkv_plan *plan, Side *src, Side *dst, int *H, int *row_bytes,
                        int *vec_bytes, int *num_layers, int *device);
 int report_cuda_error(cudaError_t e, const char *what);
+int plan_num_layers(const pdkv_plan *plan);
 
 }  // namespace pdkv

@@ -351,3 +351,14 @@ def gather_blocks(pool, geom: Geometry, ids):
     idx = np.asarray(ids, np.int64)
     out = v[idx] if geom.layout == BLOCK_MAJOR else v[:, :, idx]
     return np.ascontiguousarray(out).reshape(-1)
+
+
+def slice_batch(b: Batch, r0: int, r1: int) -> Batch:
+    """Requests [r0, r1) of a batch as a batch of their own (same block ids)."""
+    def cut(off, tbl):
+        return (off[r0:r1 + 1] - off[r0]).astype(np.int64), tbl[off[r0]:off[r1]].copy()
+
+    s_off, s_tbl = cut(b.src_tbl_off, b.src_tbl)
+    d_off, d_tbl = cut(b.dst_tbl_off, b.dst_tbl)
+    skip = None if b.dst_skip is None else b.dst_skip[b.dst_tbl_off[r0]:b.dst_tbl_off[r1]].copy()
+    return Batch(b.seq_len[r0:r1].copy(), s_off, s_tbl, d_off, d_tbl, skip)
