@@ -490,16 +490,37 @@ def e2e_leg(args, w, src_t, dst_t, buf_t, stream, step_bytes, torch, B, Transfer
     steps = max(1, min(args.e2e_steps, args.steps))
     up_down = [0, 0]
 
+    # The batch is cut into request groups that go round three streams, so that one
+    # group's download overlaps the next group's upload (PCIe is full duplex) and
+    # the kernels in between.  Every group runs the whole step for its requests.
+    from paper_2408_08147_b200 import workloads as W
+
+    n_groups = max(1, min(args.e2e_groups, w.batch.n_req))
+    cuts = [round(i * w.batch.n_req / n_groups) for i in range(n_groups + 1)]
+    groups = [W.slice_batch(w.batch, cuts[i], cuts[i + 1]) for i in range(n_groups)]
+    streams = [torch.cuda.Stream() for _ in range(min(3, n_groups))]
+    setup = torch.cuda.Stream()
+
     def one():
-        s = TransferSession(w.src, src_t, w.dst, dst_t, w.batch, stream.cuda_stream)
-        s.upload_blocks(h_src)          # pdkv_upload_blocks: H2D of every referenced prefill block
-        s.pack(buf_t)
-        s.unpack(buf_t)
-        s.transfer()
-        s.download_blocks(h_dst)        # pdkv_download_blocks: D2H of every written decode block
-        stream.synchronize()
-        up_down[:] = s.block_bytes()
-        s.close()
+        sessions, at, up, down = [], 0, 0, 0
+        for g, part in enumerate(groups):
+            st = streams[g % len(streams)].cuda_stream
+            s = TransferSession(w.src, src_t, w.dst, dst_t, part, setup.cuda_stream)   # plan: tables from host
+            piece = buf_t[at:at + s.buffer_bytes] if s.buffer_bytes else buf_t[:16]
+            at += s.buffer_bytes
+            s.upload_blocks(h_src, st)      # pdkv_upload_blocks: H2D of the group's prefill blocks
+            s.pack(piece, stream=st)
+            s.unpack(piece, stream=st)
+            s.transfer(stream=st)
+            s.download_blocks(h_dst, st)    # pdkv_download_blocks: D2H of the group's decode blocks
+            a, b = s.block_bytes()
+            up, down = up + a, down + b
+            sessions.append(s)
+        for st in streams:
+            st.synchronize()
+        up_down[:] = [up, down]
+        for s in sessions:
+            s.close()
 
     one()
     barrier()
@@ -516,7 +537,8 @@ def e2e_leg(args, w, src_t, dst_t, buf_t, stream, step_bytes, torch, B, Transfer
             "h2d_bytes_per_step": int(up_down[0]), "d2h_bytes_per_step": int(up_down[1]),
             "includes": "pdkv_plan_create (tables from host arrays), pdkv_upload_blocks from a pinned host image of "
                         "the prefill pool, pack, unpack, fused, pdkv_download_blocks into a pinned host image of "
-                        "the decode pool; wall clock"}
+                        "the decode pool; wall clock",
+            "pipeline": f"{n_groups} request groups over {len(streams)} streams"}
 
 
 def overlap_arm(args):
@@ -604,6 +626,59 @@ def overlap_arm(args):
     print(json.dumps(out), flush=True)
 
 
+def retrieval_arm(args):
+    """Asynchronous retrieval (Sec. 3.5): the batch arrives as request groups that
+    are retrieved through a queue of `capacity` receive slots.  Reports makespan
+    and mean completion time for capacities 1 (one after another) to 4
+    (several transmissions sharing the bandwidth)."""
+    import torch
+
+    from paper_2408_08147_b200 import binding as B
+    from paper_2408_08147_b200 import workloads as W
+
+    B.lib()
+    torch.cuda.set_device(0)
+    w = W.make_config(args.config)
+    src_t, dst_t = alloc_pools(w, torch)
+    torch.cuda.synchronize()
+    ps = B.pdkv_pool_create(B.desc_of(w.src), src_t.data_ptr(), src_t.numel(), 0)
+    pd = B.pdkv_pool_create(B.desc_of(w.dst), dst_t.data_ptr(), dst_t.numel(), 0)
+    n_groups = max(1, min(args.e2e_groups, w.batch.n_req))
+    cuts = [round(i * w.batch.n_req / n_groups) for i in range(n_groups + 1)]
+    groups = [W.slice_batch(w.batch, cuts[i], cuts[i + 1]) for i in range(n_groups)]
+    out = {"mode": "retrieval", "config": {"workload": workload_name(w), "groups": n_groups}, "capacities": {}}
+    for cap in (1, 2, 4):
+        q = B.pdkv_queue_create(ps, pd, 0, cap)
+        best = None
+        for _ in range(max(3, args.steps // 10)):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            pending, done_at = [], []
+            for part in groups:
+                while True:
+                    t = B.pdkv_queue_submit(q, part.seq_len, part.src_tbl_off, part.src_tbl, part.dst_tbl_off,
+                                            part.dst_tbl, part.dst_skip)
+                    if t is not None:
+                        pending.append(t)
+                        break
+                    B.pdkv_queue_wait(q, pending[0])
+                    done_at.append(time.perf_counter() - t0)
+                    B.pdkv_queue_release(q, pending.pop(0))
+            for t in pending:
+                B.pdkv_queue_wait(q, t)
+                done_at.append(time.perf_counter() - t0)
+                B.pdkv_queue_release(q, t)
+            rec = {"makespan_ms": done_at[-1] * 1e3, "mean_completion_ms": statistics.fmean(done_at) * 1e3}
+            if best is None or rec["makespan_ms"] < best["makespan_ms"]:
+                best = rec
+        best["rejected_submits"] = B.pdkv_queue_stats(q)[3]
+        out["capacities"][str(cap)] = best
+        B.pdkv_queue_destroy(q)
+    B.pdkv_pool_destroy(ps)
+    B.pdkv_pool_destroy(pd)
+    print(json.dumps(out), flush=True)
+
+
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -617,10 +692,12 @@ def parse():
     ap.add_argument("--layouts", default="", help="two letters, e.g. AB: prefill block-major, decode layer-major")
     ap.add_argument("--tune", nargs=2, action="append", metavar=("KEY", "VALUE"))
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-groups", type=int, default=8, help="request groups pipelined over three streams in the e2e leg")
     ap.add_argument("--no-extras", action="store_true", help="skip baseline, e2e and CPU legs")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--overlap", action="store_true", help="per-layer transfer overlapped with a compute stand-in")
+    ap.add_argument("--retrieval", action="store_true", help="request groups through the asynchronous retrieval queue")
     ap.add_argument("--gemm-n", type=int, default=4096)
     ap.add_argument("--side-priority", type=int, default=1, help="1: transfer stream has high priority")
     ap.add_argument("--no-blockwise", action="store_true")
@@ -632,6 +709,8 @@ if __name__ == "__main__":
     a.warmup = max(a.warmup, 3) if a.impl == "pdkv" else a.warmup
     if a.overlap:
         overlap_arm(a)
+    elif a.retrieval:
+        retrieval_arm(a)
     elif a.impl == "reference":
         reference_arm(a)
     else:

@@ -510,10 +510,9 @@ int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip_gr
         // one device allocation: [status words][pack tiles][unpack tiles][transfer tiles]
         DeviceGuard guard(pl->device);
         if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
-        cudaDeviceProp prop;
-        cudaError_t e = cudaGetDeviceProperties(&prop, pl->device);
-        if (e != cudaSuccess) return cuda_fail(e, "cudaGetDeviceProperties");
-        pl->sm_count = prop.multiProcessorCount;
+        // (cudaGetDeviceProperties costs milliseconds; one attribute query does not)
+        cudaError_t e = cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, pl->device);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
         const size_t head = 256;
         size_t total = head;
         for (int op = 0; op < 3; ++op) total += pl->tiles[op].size() * sizeof(Tile);
