@@ -292,11 +292,14 @@ int pdkv_plan_tiles(const pdkv_plan *plan, int op, const pdkv_tile **tiles, int6
 int pdkv_plan_status(const pdkv_plan *plan, void *stream);
 
 /* Process-wide tunables, read when a plan is created or a call is launched:
- *   "tile_bytes"     target bytes moved per tile (default 65536)
- *   "ctas_per_sm"    persistent CTAs per SM (default 4)
- *   "threads"        threads per CTA, multiple of 32 (default 256; clamped to
- *                    what the register budget of the chosen variant allows)
- *   "unroll"         independent accesses in flight per thread: 1, 2, 4, 8 (default 1)
+ *   "tile_bytes"     target bytes moved per tile (default 32768)
+ *   "ctas_per_sm"    persistent CTAs per SM (default 2)
+ *   "threads"        threads per CTA, multiple of 32, clamped to what the register
+ *                    budget of the chosen variant allows; 0 = automatic (default)
+ *   "unroll"         independent accesses in flight per thread: 1, 2, 4, 8;
+ *                    0 = automatic (default).  Automatic means 512 threads x 1
+ *                    access for flat copies (token-major on both sides) and
+ *                    256 threads x 4 for copies with a head-major side
  *   "vec32"          1: use 32-byte accesses when rows and bases allow (default 1)
  *   "lc_fastest"     1: consecutive work items walk the (layer, K/V) strips of
  *                    one tile; 0: they walk the tiles of one strip (default 0)

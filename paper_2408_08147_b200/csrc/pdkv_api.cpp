@@ -257,6 +257,15 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     cfg.sm_count = pl->sm_count;
     cfg.variant = (int)pdkv::tunables().variant;
     cfg.check_bounds = pdkv::tunables().debug_bounds != 0;
+    {   // automatic launch shape, measured best per class of copy on B200: a flat copy
+        // (token-major on both sides) runs 512 threads with one access in flight each, a
+        // row-permuting or head-major copy 256 threads with four, i.e. one 32 KiB tile per pass
+        const int64_t hrow = pl->hrow_bytes, row = pl->row_bytes;
+        const bool flat = src.head_stride == row && src.tok_stride == hrow && dst.head_stride == row &&
+                          dst.tok_stride == hrow;
+        if (cfg.unroll == 0) cfg.unroll = flat ? 1 : 4;
+        if (cfg.threads == 0) cfg.threads = flat ? 512 : 256;
+    }
     cfg.stages = (int)pdkv::tunables().stages;
     cfg.max_tile_bytes = pl->max_tile_bytes;
     cudaError_t e;
@@ -751,8 +760,8 @@ int pdkv_tune(const char *key, int64_t value)
     const std::string k(key);
     if (k == "tile_bytes" && value >= 1 && value <= (1ll << 30)) t.tile_bytes = value;
     else if (k == "ctas_per_sm" && value >= 1 && value <= 32) t.ctas_per_sm = value;
-    else if (k == "threads" && value >= 32 && value <= 1024 && value % 32 == 0) t.threads = value;
-    else if (k == "unroll" && (value == 1 || value == 2 || value == 4 || value == 8)) t.unroll = value;
+    else if (k == "threads" && (value == 0 || (value >= 32 && value <= 1024 && value % 32 == 0))) t.threads = value;
+    else if (k == "unroll" && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8)) t.unroll = value;
     else if (k == "vec32" && (value == 0 || value == 1)) t.vec32 = value;
     else if (k == "lc_fastest" && (value == 0 || value == 1)) t.lc_fastest = value;
     else if (k == "chunked" && (value == 0 || value == 1)) t.chunked = value;

@@ -62,10 +62,10 @@ cudaError_t launch_bulk(const CopyParams &p, const LaunchConfig &cfg, cudaStream
 bool bulk_supported(const LaunchConfig &cfg, int row_bytes);
 
 struct Tunables {
-    int64_t tile_bytes = 65536;
-    int64_t ctas_per_sm = 4;
-    int64_t threads = 256;
-    int64_t unroll = 1;
+    int64_t tile_bytes = 32768;
+    int64_t ctas_per_sm = 2;
+    int64_t threads = 0;   // 0: chosen with unroll, per class of copy
+    int64_t unroll = 0;    // 0: chosen per class of copy
     int64_t vec32 = 1;
     int64_t lc_fastest = 0;
     int64_t chunked = 0;

@@ -109,8 +109,8 @@ extern "C" int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
         if (vec_bytes == 16 && t.vec32 && row_bytes % 32 == 0 &&
             ((reinterpret_cast<uintptr_t>(p.src.base) | reinterpret_cast<uintptr_t>(p.dst.base)) & 31u) == 0)
             cfg.vec_bytes = 32;
-        cfg.unroll = (int)t.unroll;
-        cfg.threads = (int)t.threads;
+        cfg.unroll = t.unroll ? (int)t.unroll : 4;
+        cfg.threads = t.threads ? (int)t.threads : 256;
         cfg.ctas_per_sm = (int)t.ctas_per_sm;
         cfg.sm_count = slot.sm_count;
         cfg.variant = 0;

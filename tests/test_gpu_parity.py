@@ -23,7 +23,7 @@ def _gpu_lib():
     B.pdkv_tune("debug_bounds", 0)
     yield
     B.pdkv_tune("debug_bounds", 0)
-    B.pdkv_tune("tile_bytes", 65536)
+    B.pdkv_tune("tile_bytes", 32768)
     B.pdkv_tune("lc_fastest", 0)
     B.pdkv_tune("variant", 0)
     B.pdkv_tune("stages", 3)
@@ -120,7 +120,7 @@ def test_tile_size_and_work_order_do_not_change_the_result(oracle, tile_bytes, l
         check_all_ops(oracle, W.make_config(3, num_layers=2, n_req=8, max_len=1200))
         check_all_ops(oracle, W.make_config(5, num_layers=1, n_req=30, src_block=32))
     finally:
-        B.pdkv_tune("tile_bytes", 65536)
+        B.pdkv_tune("tile_bytes", 32768)
         B.pdkv_tune("lc_fastest", 0)
 
 
@@ -149,7 +149,7 @@ def test_bulk_copy_variant(oracle, stages, tile_bytes, chunked):
     finally:
         B.pdkv_tune("variant", 0)
         B.pdkv_tune("stages", 3)
-        B.pdkv_tune("tile_bytes", 65536)
+        B.pdkv_tune("tile_bytes", 32768)
         B.pdkv_tune("chunked", 0)
 
 

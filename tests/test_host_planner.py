@@ -22,7 +22,7 @@ def built():
     B.pdkv_tune("dry_run", 1)
     yield
     B.pdkv_tune("dry_run", 0)
-    B.pdkv_tune("tile_bytes", 65536)
+    B.pdkv_tune("tile_bytes", 32768)
 
 
 def test_library_exports_every_declared_symbol():
@@ -153,6 +153,7 @@ def test_launch_argument_errors_and_dry_run_refusal():
         B.pdkv_tune("no_such_key", 1)
     with pytest.raises(B.PdkvError):
         B.pdkv_tune("threads", 33)
+    B.pdkv_tune("threads", 0)
 
 
 # --------------------------------------------------------------------------

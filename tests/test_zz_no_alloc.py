@@ -57,7 +57,7 @@ def test_noalloc_matches_plan_based_transfer_twice_in_a_row():
         pytest.skip("no CUDA device")
     B.lib()
     B.pdkv_tune("dry_run", 0)
-    B.pdkv_tune("tile_bytes", 65536)
+    B.pdkv_tune("tile_bytes", 32768)
     stream = torch.cuda.Stream()
     # call 1: many tiles, re-blocking 16 -> 128, block-major -> layer-major
     first = W.make_config(3, num_layers=2, n_req=10, max_len=1500)
@@ -98,7 +98,7 @@ def test_noalloc_rejects_batches_beyond_the_scratch_limit():
                                     b.dst_tbl, b.dst_skip, 0, 2)    # layer range outside the model
         assert e.value.status in (B.PDKV_ERR_INVALID_ARG, B.PDKV_ERR_LIMIT)
     finally:
-        B.pdkv_tune("tile_bytes", 65536)
+        B.pdkv_tune("tile_bytes", 32768)
         B.pdkv_pool_destroy(ps)
         B.pdkv_pool_destroy(pd)
     torch.cuda.synchronize()
