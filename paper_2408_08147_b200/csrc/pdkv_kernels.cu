@@ -123,8 +123,18 @@ copy_tiles_kernel(const CopyParams p)
         w_end = n_work;
         w_step = gridDim.x;
     }
+    const bool narrow = n_work <= 0xFFFFFFFFll;   // 32-bit divisions are several times cheaper
     auto split = [&](int64_t x, int32_t &ti, int32_t &lci) {
-        if (p.lc_fastest) {
+        if (narrow) {
+            const uint32_t x32 = (uint32_t)x;
+            if (p.lc_fastest) {
+                ti = (int32_t)(x32 / (uint32_t)p.n_lc);
+                lci = (int32_t)(x32 - (uint32_t)ti * (uint32_t)p.n_lc);
+            } else {
+                lci = (int32_t)(x32 / (uint32_t)p.n_tiles);
+                ti = (int32_t)(x32 - (uint32_t)lci * (uint32_t)p.n_tiles);
+            }
+        } else if (p.lc_fastest) {
             ti = (int32_t)(x / p.n_lc);
             lci = (int32_t)(x - (int64_t)ti * p.n_lc);
         } else {
