@@ -187,16 +187,16 @@ def alloc_pools(w, torch, seed_offset=0):
 def token_major_torch(geom, pool_t, tbl, length, torch):
     """[L][2][len][H][D] view-copy of one request, through reshape/index/permute
     (an independent cross-check of the kernels; not the CPU checker)."""
-    v = pool_t.view(torch.int16).view(geom.shape())
+    v = pool_t.view(torch.uint8).view(*geom.shape(), geom.elem_bytes)   # last axis: the bytes of one element
     B = geom.block_tokens
     nb = -(-length // B)
     idx = torch.as_tensor(tbl[:nb].astype("int64"), device=pool_t.device)
     if geom.layout == 0:
-        x = v[idx].permute(1, 2, 0, 3, 4, 5)
+        x = v[idx].permute(1, 2, 0, 3, 4, 5, 6)
     else:
-        x = v[:, :, idx].permute(0, 1, 2, 4, 3, 5)
+        x = v[:, :, idx].permute(0, 1, 2, 4, 3, 5, 6)
     L, H, D = geom.num_layers, geom.num_kv_heads, geom.head_dim
-    return x.reshape(L, 2, nb * B, H, D)[:, :, :length]
+    return x.reshape(L, 2, nb * B, H, D * geom.elem_bytes)[:, :, :length]
 
 
 def sanity_check(w, src_t, dst_t, torch) -> bool:
@@ -256,6 +256,8 @@ def cpu_baseline(w, src_t, budget_s=20.0):
     from oracle import pdkv_oracle as O
     from paper_2408_08147_b200 import workloads as W
 
+    if w.src.elem_bytes != 2:
+        return {"value": None, "unit": UNIT, "kind": "oracle", "skipped": "CPU leg is wired for 2-byte elements"}
     cores = os.cpu_count() or 1
     n = min(w.batch.n_req, cores, 8)
     # keep the sample near `budget_s` CPU-seconds at ~0.4 GB/s per thread
@@ -352,6 +354,10 @@ def main_arm(args):
         kw["src_block"] = args.src_block
     if args.n_req:
         kw["n_req"] = args.n_req
+    if args.elem_bytes:
+        kw["elem_bytes"] = args.elem_bytes
+    if args.kv_heads:
+        kw["num_kv_heads"] = args.kv_heads
     if args.num_layers:
         kw["num_layers"] = args.num_layers
     if args.layouts:
@@ -481,9 +487,12 @@ def e2e_leg(args, w, src_t, dst_t, buf_t, stream, step_bytes, torch, B, Transfer
         free_host = psutil.virtual_memory().available
     except Exception:
         pass
-    need = src_t.numel() + dst_t.numel()
-    if free_host is not None and need > 0.6 * free_host:
-        return {"value": None, "unit": UNIT, "skipped": f"needs {need >> 30} GiB pinned host memory"}
+    _, _, world = dist_env()
+    need = (src_t.numel() + dst_t.numel()) * world      # every rank on this node pins its own images
+    if free_host is not None and need > 0.5 * free_host:
+        return {"value": None, "unit": UNIT,
+                "skipped": f"needs {need >> 30} GiB of pinned host memory across {world} ranks, "
+                           f"{free_host >> 30} GiB available"}
     h_src = torch.empty(src_t.numel(), dtype=torch.uint8, pin_memory=True)
     h_dst = torch.empty(dst_t.numel(), dtype=torch.uint8, pin_memory=True)
     h_src.copy_(src_t)
@@ -687,6 +696,8 @@ def parse():
     ap.add_argument("--impl", default="pdkv", choices=["pdkv", "reference"])
     ap.add_argument("--config", type=int, default=2, help="workload 1..5 (2 = the headline config)")
     ap.add_argument("--src-block", type=int, default=0)
+    ap.add_argument("--elem-bytes", type=int, default=0, help="KV element size override (1 = fp8/int8 KV)")
+    ap.add_argument("--kv-heads", type=int, default=0, help="KV head count override (1 = MQA)")
     ap.add_argument("--n-req", type=int, default=0, help="shrink the batch (profiling captures)")
     ap.add_argument("--num-layers", type=int, default=0, help="shrink the model (profiling captures)")
     ap.add_argument("--layouts", default="", help="two letters, e.g. AB: prefill block-major, decode layer-major")

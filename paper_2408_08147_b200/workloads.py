@@ -184,7 +184,9 @@ def build_workload(name: str, seed: int, *, num_layers: int, num_kv_heads: int,
 
 def make_config(idx: int, *, num_layers: Optional[int] = None, n_req: Optional[int] = None,
                 src_block: Optional[int] = None, src_layout: Optional[int] = None,
-                dst_layout: Optional[int] = None, max_len: Optional[int] = None) -> Workload:
+                dst_layout: Optional[int] = None, max_len: Optional[int] = None,
+                elem_bytes: Optional[int] = None, num_kv_heads: Optional[int] = None,
+                head_dim: Optional[int] = None) -> Workload:
     """The five benchmark workloads (idx 1..5); keyword overrides shrink them.
 
     1 tiny; 2 8B-shaped uniform, same layout both sides; 3 8B-shaped lognormal
@@ -195,8 +197,8 @@ def make_config(idx: int, *, num_layers: Optional[int] = None, n_req: Optional[i
     if idx == 1:
         n = n_req or 8
         lens = draw_lengths("uniform", n, seed, lo=1, hi=max_len or 300)
-        return build_workload("tiny", seed, num_layers=num_layers or 2, num_kv_heads=4,
-                              head_dim=64, elem_bytes=2, seq_len=lens,
+        return build_workload("tiny", seed, num_layers=num_layers or 2, num_kv_heads=num_kv_heads or 4,
+                              head_dim=head_dim or 64, elem_bytes=elem_bytes or 2, seq_len=lens,
                               src_layout=BLOCK_MAJOR if src_layout is None else src_layout,
                               src_block=src_block or 16,
                               dst_layout=LAYER_MAJOR if dst_layout is None else dst_layout,
@@ -206,7 +208,8 @@ def make_config(idx: int, *, num_layers: Optional[int] = None, n_req: Optional[i
         lens = draw_lengths("fixed", n, seed, value=max_len or 2048)
         lay = BLOCK_MAJOR if src_layout is None else src_layout
         return build_workload("llama3-8b-uniform", seed, num_layers=num_layers or 32,
-                              num_kv_heads=8, head_dim=128, elem_bytes=2, seq_len=lens,
+                              num_kv_heads=num_kv_heads or 8, head_dim=head_dim or 128, elem_bytes=elem_bytes or 2,
+                              seq_len=lens,
                               src_layout=lay, src_block=src_block or 128,
                               dst_layout=lay if dst_layout is None else dst_layout,
                               dst_block=128)
@@ -215,8 +218,8 @@ def make_config(idx: int, *, num_layers: Optional[int] = None, n_req: Optional[i
         lens = draw_lengths("lognormal", n, seed, median=1024, sigma=0.8, lo=16,
                             hi=max_len or 8192)
         return build_workload("llama3-8b-lognormal-reblock", seed,
-                              num_layers=num_layers or 32, num_kv_heads=8, head_dim=128,
-                              elem_bytes=2, seq_len=lens,
+                              num_layers=num_layers or 32, num_kv_heads=num_kv_heads or 8,
+                              head_dim=head_dim or 128, elem_bytes=elem_bytes or 2, seq_len=lens,
                               src_layout=BLOCK_MAJOR if src_layout is None else src_layout,
                               src_block=src_block or 16,
                               dst_layout=LAYER_MAJOR if dst_layout is None else dst_layout,
@@ -225,7 +228,8 @@ def make_config(idx: int, *, num_layers: Optional[int] = None, n_req: Optional[i
         n = n_req or 16
         lens = draw_lengths("fixed", n, seed, value=max_len or 4096)
         return build_workload("llama3-70b-fragmented", seed, num_layers=num_layers or 80,
-                              num_kv_heads=8, head_dim=128, elem_bytes=2, seq_len=lens,
+                              num_kv_heads=num_kv_heads or 8, head_dim=head_dim or 128, elem_bytes=elem_bytes or 2,
+                              seq_len=lens,
                               src_layout=BLOCK_MAJOR if src_layout is None else src_layout,
                               src_block=src_block or 64,
                               dst_layout=LAYER_MAJOR if dst_layout is None else dst_layout,
@@ -234,7 +238,8 @@ def make_config(idx: int, *, num_layers: Optional[int] = None, n_req: Optional[i
         n = n_req or 1024
         lens = draw_lengths("uniform", n, seed, lo=64, hi=max_len or 512)
         return build_workload("tidal-small-requests", seed, num_layers=num_layers or 32,
-                              num_kv_heads=8, head_dim=128, elem_bytes=2, seq_len=lens,
+                              num_kv_heads=num_kv_heads or 8, head_dim=head_dim or 128, elem_bytes=elem_bytes or 2,
+                              seq_len=lens,
                               src_layout=BLOCK_MAJOR if src_layout is None else src_layout,
                               src_block=src_block or 16,
                               dst_layout=LAYER_MAJOR if dst_layout is None else dst_layout,
