@@ -426,14 +426,15 @@ def main_arm(args):
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-           "scaling": "weak", "vs_baseline": None, "dtype": "u16", "data": "synthetic",
+           "scaling": "weak", "vs_baseline": None, "dtype": f"u{8 * w.src.elem_bytes}", "data": "synthetic",
            "config": {"workload": workload_name(w), "config_index": args.config,
                       "step": "pdkv_pack + pdkv_unpack + pdkv_transfer, all layers",
                       "payload_bytes": sess.buffer_bytes, "step_bytes": step_bytes,
                       "l2": "inputs exceed L2 (pools and buffer are GiB-sized; no flush needed)"
                       if sess.buffer_bytes > (1 << 29) else "L2-resident workload: not an HBM number",
                       "tunables": {k: B.pdkv_tune_get(k) for k in
-                                   ("tile_bytes", "ctas_per_sm", "threads", "unroll", "vec32", "lc_fastest", "variant")}},
+                                   ("tile_bytes", "ctas_per_sm", "threads", "unroll", "group_threads", "vec32", "lc_fastest",
+                                    "variant")}},
            "ops": per_op, "roofline": roofline, "gpu_launches": launches_per_step * args.steps,
            "sanity_check": "ok" if ok else "MISMATCH", "clocks": clk.summary()}
 

@@ -300,6 +300,10 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream);
  *                    0 = automatic (default).  Automatic means 512 threads x 1
  *                    access for flat copies (token-major on both sides) and
  *                    256 threads x 4 for copies with a head-major side
+ *   "group_threads"  threads that cooperate on one work item (a CTA hosts
+ *                    threads / group_threads independent groups); 0 = automatic
+ *                    (default): sized so that the plan's mean tile is covered in
+ *                    one or two passes, 32 at least
  *   "vec32"          1: use 32-byte accesses when rows and bases allow (default 1)
  *   "lc_fastest"     1: consecutive work items walk the (layer, K/V) strips of
  *                    one tile; 0: they walk the tiles of one strip (default 0)

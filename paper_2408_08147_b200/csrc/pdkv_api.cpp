@@ -94,6 +94,7 @@ struct pdkv_plan {
     unsigned long long *dev_status = nullptr;
     int vec_bytes = 16;
     int64_t max_tile_bytes = 0;
+    int64_t mean_tile_bytes[3] = {0, 0, 0};   // per operation, over its tile list
     int sm_count = 1;
     int lc_fastest = 1;
 };
@@ -265,6 +266,16 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
                           dst.tok_stride == hrow;
         if (cfg.unroll == 0) cfg.unroll = flat ? 1 : 4;
         if (cfg.threads == 0) cfg.threads = flat ? 512 : 256;
+        // threads per work item: a flat tile is covered in two passes, any other in one, so
+        // that batches of small tiles (few KV heads, small blocks) still fill the CTA
+        cfg.group_threads = (int)pdkv::tunables().group_threads;
+        if (cfg.group_threads == 0) {
+            const int64_t vecs = std::max<int64_t>(1, pl->mean_tile_bytes[op] / cfg.vec_bytes);
+            const int64_t want = vecs / (flat ? 2 : cfg.unroll);
+            int g = 32;
+            while (g < want && g < cfg.threads) g *= 2;
+            cfg.group_threads = g;
+        }
     }
     cfg.stages = (int)pdkv::tunables().stages;
     cfg.max_tile_bytes = pl->max_tile_bytes;
@@ -506,8 +517,12 @@ int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip_gr
         if (src && dst) build_tiles(*pl, PDKV_OP_TRANSFER, *batch, cap_tok);
         for (int op = 0; op < 3; ++op) {
             if (pl->tiles[op].size() > (size_t)INT32_MAX) return PDKV_ERR_INVALID_ARG;
-            for (const Tile &t : pl->tiles[op])
+            int64_t sum = 0;
+            for (const Tile &t : pl->tiles[op]) {
                 pl->max_tile_bytes = std::max<int64_t>(pl->max_tile_bytes, t.ntok * pl->hrow_bytes);
+                sum += t.ntok * pl->hrow_bytes;
+            }
+            pl->mean_tile_bytes[op] = pl->tiles[op].empty() ? 0 : sum / (int64_t)pl->tiles[op].size();
         }
 
         if (pdkv::tunables().dry_run || g_host_only_plan) {  // host-only plan: tile lists can be inspected, nothing can launch
@@ -765,6 +780,7 @@ int pdkv_tune(const char *key, int64_t value)
     else if (k == "vec32" && (value == 0 || value == 1)) t.vec32 = value;
     else if (k == "lc_fastest" && (value == 0 || value == 1)) t.lc_fastest = value;
     else if (k == "chunked" && (value == 0 || value == 1)) t.chunked = value;
+    else if (k == "group_threads" && (value == 0 || (value >= 32 && value <= 1024 && value % 32 == 0))) t.group_threads = value;
     else if (k == "debug_bounds" && (value == 0 || value == 1)) t.debug_bounds = value;
     else if (k == "variant" && value >= 0 && value <= 1) t.variant = value;
     else if (k == "stages" && value >= 2 && value <= 16) t.stages = value;
@@ -785,6 +801,7 @@ int pdkv_tune_get(const char *key, int64_t *value)
     else if (k == "vec32") *value = t.vec32;
     else if (k == "lc_fastest") *value = t.lc_fastest;
     else if (k == "chunked") *value = t.chunked;
+    else if (k == "group_threads") *value = t.group_threads;
     else if (k == "debug_bounds") *value = t.debug_bounds;
     else if (k == "variant") *value = t.variant;
     else if (k == "stages") *value = t.stages;

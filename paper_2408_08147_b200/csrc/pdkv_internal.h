@@ -38,13 +38,15 @@ struct CopyParams {
     int32_t H;
     int32_t row_bytes;   // D * E
     int32_t lc_fastest;
-    int32_t chunked;     // 1: each CTA takes one contiguous run of work items
+    int32_t chunked;     // 1: each group takes one contiguous run of work items
+    int32_t group_threads;  // threads that cooperate on one work item (set by the launcher)
     unsigned long long *status;  // [0] != 0: an access was refused; [1] offending offset
 };
 
 struct LaunchConfig {
     int vec_bytes;   // 32, 16, 8, 4, 2 or 1
     int unroll;      // independent accesses per thread: 1, 2, 4 or 8
+    int group_threads;  // threads per work item; the launcher rounds it to a divisor of `threads`
     int threads;
     int ctas_per_sm;
     int sm_count;
@@ -68,6 +70,7 @@ struct Tunables {
     int64_t unroll = 0;    // 0: chosen per class of copy
     int64_t vec32 = 1;
     int64_t lc_fastest = 0;
+    int64_t group_threads = 0;   // 0: sized from the plan's mean tile
     int64_t chunked = 0;
     int64_t debug_bounds = 0;
     int64_t variant = 0;

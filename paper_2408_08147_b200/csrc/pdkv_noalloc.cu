@@ -114,6 +114,7 @@ extern "C" int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
         cfg.ctas_per_sm = (int)t.ctas_per_sm;
         cfg.sm_count = slot.sm_count;
         cfg.variant = 0;
+        cfg.group_threads = cfg.threads;
         cfg.stages = 0;
         cfg.max_tile_bytes = 0;
         cfg.check_bounds = false;
