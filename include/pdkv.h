@@ -22,7 +22,9 @@
  *     small device arrays (tile lists), freed by pdkv_plan_destroy().
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *     stream).  pack / unpack / transfer only enqueue work: no allocation, no
- *     host<->device copy, no synchronisation.
+ *     host<->device copy, no synchronisation; after one call outside capture
+ *     they can be recorded into a CUDA graph (e.g. the per-layer sequence of a
+ *     model) and replayed.
  *   - Elements are opaque: `elem_bytes` bytes are moved bit for bit (NaN
  *     payloads and -0 survive).
  *

@@ -281,3 +281,43 @@ def test_host_resident_pools(oracle, idx, kw):
     assert up <= w.src.num_bytes() and down <= w.dst.num_bytes()
     if w.src_occupied.size or w.batch.dst_skip is not None:
         assert up < w.src.num_bytes()
+
+
+def test_per_layer_calls_replayed_from_a_cuda_graph(oracle):
+    """pack / unpack / transfer only enqueue kernels (no allocation, copy or
+    synchronisation), so a per-layer sequence can be captured once and replayed."""
+    from paper_2408_08147_b200.session import TransferSession
+
+    w = W.make_config(3, num_layers=4, n_req=6, max_len=700)
+    src = W.fill_pool_numpy(w.src, w.seed)
+    sent = W.sentinel_pool_numpy(w.dst)
+    want = sent.copy()
+    oracle.transfer(w.src, src, w.dst, want, w.batch)
+    src_t, dst_t = dev(src), dev(sent)
+    cap = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with TransferSession(w.src, src_t, w.dst, dst_t, w.batch, cap.cuda_stream) as s:
+        buf_t = torch.zeros(s.buffer_bytes, dtype=torch.uint8, device="cuda")
+        s.transfer((0, 1))                      # warm-up outside capture (module load, attributes)
+        s.pack(buf_t, (0, 1)); s.unpack(buf_t, (0, 1))
+        torch.cuda.synchronize()
+        dst_t.copy_(dev(sent))
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=cap):
+            st = torch.cuda.current_stream().cuda_stream
+            for l in range(2):
+                s.transfer((l, l + 1), st)
+            for l in range(2, 4):
+                s.pack(buf_t, (l, l + 1), st)
+                s.unpack(buf_t, (l, l + 1), st)
+        torch.cuda.synchronize()
+        assert np.array_equal(host(dst_t), sent), "capture must not execute anything"
+        graph.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(host(dst_t), want)
+        dst_t.copy_(dev(sent))
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(host(dst_t), want)
