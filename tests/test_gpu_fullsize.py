@@ -1,9 +1,10 @@
 """GPU parity at the benchmark's full sizes, in the launch configuration the
 benchmark times (library defaults).  Pools of 8-50 GiB cannot be replayed on the
-CPU checker in full, so a seeded sample of requests is checked bit for bit:
-each sampled request becomes a self-contained sub-problem (its blocks gathered
-out of both pools), the checker computes buffer and decode blocks for it, and
-the GPU's bytes for that request must be identical.  Bytes nobody may touch
+CPU checker in one piece, so requests are checked as self-contained sub-problems
+(their blocks gathered out of both pools): the checker computes buffer and
+decode blocks for the sub-problem and the GPU's bytes for those requests must be
+identical.  Configs 2 and 3 are checked in full this way (every request, hence
+every owned byte); configs 4 and 5 on a seeded sample of requests.  Bytes nobody may touch
 (resident decode blocks, the buffer's slack) are compared with the sentinel."""
 import numpy as np
 import pytest
@@ -38,7 +39,9 @@ def _np16(t):
     return t.cpu().numpy().view(np.uint16)
 
 
-def run_fullsize(oracle, w, n_sample, seed):
+def run_fullsize(oracle, w, n_sample, seed, group=1):
+    """n_sample = 0 checks every request (in groups of `group` consecutive
+    requests, one checker thread each); otherwise a seeded sample."""
     from paper_2408_08147_b200.session import TransferSession
 
     import gc
@@ -51,7 +54,10 @@ def run_fullsize(oracle, w, n_sample, seed):
         pytest.skip(f"needs {need >> 30} GiB of device memory")
     b = w.batch
     rng = np.random.default_rng(seed)
-    sample = sorted({0, b.n_req - 1, *rng.integers(0, b.n_req, size=max(0, n_sample - 2)).tolist()})
+    if n_sample == 0:
+        groups = [list(range(i, min(i + group, b.n_req))) for i in range(0, b.n_req, group)]
+    else:
+        groups = [[r] for r in sorted({0, b.n_req - 1, *rng.integers(0, b.n_req, size=max(0, n_sample - 2)).tolist()})]
 
     src_t = torch.empty(w.src.num_bytes(), dtype=torch.uint8, device="cuda")
     W.fill_pool_torch(src_t, w.seed)
@@ -68,26 +74,26 @@ def run_fullsize(oracle, w, n_sample, seed):
 
         # expected bytes of every sampled request, from the checker
         expect = {}
-        for r in sample:
-            sub, s_ids, d_ids = W.compact_subproblem(w, [r])
+        for g in groups:
+            sub, s_ids, d_ids = W.compact_subproblem(w, g)
             sub_src = _np16(W.gather_blocks(src_t.view(torch.int16), w.src, s_ids))
             want_buf = np.zeros(oracle.buffer_elems(sub.batch, G, sub.src), np.uint16)
-            oracle.pack(sub.src, sub_src, sub.batch, G, want_buf)
+            oracle.pack(sub.src, sub_src, sub.batch, G, want_buf, threads=len(g))
             want_dst = W.sentinel_pool_numpy(sub.dst)
-            oracle.transfer(sub.src, sub_src, sub.dst, want_dst, sub.batch)
-            expect[r] = (want_buf, want_dst, d_ids)
-            assert want_buf.size * 2 == s.request_offsets[r + 1] - s.request_offsets[r]
+            oracle.transfer(sub.src, sub_src, sub.dst, want_dst, sub.batch, threads=len(g))
+            expect[(g[0], g[-1] + 1)] = (want_buf, want_dst, d_ids)
+            assert want_buf.size * 2 == s.request_offsets[g[-1] + 1] - s.request_offsets[g[0]]
 
         def check_dst(what):
             for r, (_, want_dst, d_ids) in expect.items():
                 got = _np16(W.gather_blocks(dst_t.view(torch.int16), w.dst, d_ids))
-                assert np.array_equal(got, want_dst), f"{what}: request {r}"
+                assert np.array_equal(got, want_dst), f"{what}: requests {r[0]}..{r[1] - 1}"
 
         s.pack(buf_t)
         torch.cuda.synchronize()
-        for r, (want_buf, _, _) in expect.items():
-            a, z = int(s.request_offsets[r]), int(s.request_offsets[r + 1])
-            assert np.array_equal(_np16(buf_t[a:z]), want_buf), f"pack: request {r}"
+        for (r0, r1), (want_buf, _, _) in expect.items():
+            a, z = int(s.request_offsets[r0]), int(s.request_offsets[r1])
+            assert np.array_equal(_np16(buf_t[a:z]), want_buf), f"pack: requests {r0}..{r1 - 1}"
         assert bool((buf_t[s.buffer_bytes:].view(torch.int16) == SENT).all()), "pack wrote past the buffer"
 
         s.unpack(buf_t)
@@ -118,16 +124,16 @@ def run_fullsize(oracle, w, n_sample, seed):
     torch.cuda.empty_cache()
 
 
-def test_config2_full_size_same_layout(oracle):
-    run_fullsize(oracle, W.make_config(2), n_sample=4, seed=2)
+def test_config2_full_size_same_layout_every_request(oracle):
+    run_fullsize(oracle, W.make_config(2), n_sample=0, seed=2, group=8)
 
 
 def test_config2_full_size_layer_major_both_sides(oracle):
     run_fullsize(oracle, W.make_config(2, src_layout=W.LAYER_MAJOR), n_sample=3, seed=22)
 
 
-def test_config3_full_size_reblocking(oracle):
-    run_fullsize(oracle, W.make_config(3), n_sample=5, seed=3)
+def test_config3_full_size_reblocking_every_request(oracle):
+    run_fullsize(oracle, W.make_config(3), n_sample=0, seed=3, group=8)
 
 
 def test_config4_full_size_70b_fragmented(oracle):
