@@ -603,10 +603,14 @@ def overlap_arm(args):
 
     results = {}
     modes = [("register copy, defaults", {"variant": 0}),
-             ("register copy, 1 CTA/SM", {"variant": 0, "ctas_per_sm": 1, "threads": 512, "unroll": 2}),
+             ("register copy on at most 64 SMs", {"variant": 0, "ctas_per_sm": 1, "threads": 1024, "unroll": 1,
+                                                  "max_ctas": 64}),
+             ("register copy on at most 32 SMs", {"variant": 0, "ctas_per_sm": 1, "threads": 1024, "unroll": 1,
+                                                  "max_ctas": 32}),
              ("bulk copy (TMA), 8 KiB tiles x 2 stages x 8 CTAs/SM",
               {"variant": 1, "tile_bytes": 8192, "stages": 2, "ctas_per_sm": 8})]
-    defaults = {k: B.pdkv_tune_get(k) for k in ("variant", "ctas_per_sm", "threads", "unroll", "tile_bytes", "stages")}
+    defaults = {k: B.pdkv_tune_get(k) for k in ("variant", "ctas_per_sm", "threads", "unroll", "tile_bytes", "stages",
+                                                "max_ctas")}
     t_compute = timed(compute_only, args.steps)
     for name, tune in modes:
         for k, v in {**defaults, **tune}.items():

@@ -296,6 +296,9 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream);
 /* Process-wide tunables, read when a plan is created or a call is launched:
  *   "tile_bytes"     target bytes moved per tile (default 32768)
  *   "ctas_per_sm"    persistent CTAs per SM (default 2)
+ *   "max_ctas"       cap on the grid size, 0 = none (default).  A small grid
+ *                    leaves most SMs to other kernels of the process at a
+ *                    proportionally lower copy rate
  *   "threads"        threads per CTA, multiple of 32, clamped to what the register
  *                    budget of the chosen variant allows; 0 = automatic (default)
  *   "unroll"         independent accesses in flight per thread: 1, 2, 4, 8;

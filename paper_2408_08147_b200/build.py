@@ -28,7 +28,7 @@ def _stale() -> bool:
     if not os.path.exists(LIB_PATH):
         return True
     t = os.path.getmtime(LIB_PATH)
-    deps = sources() + glob.glob(os.path.join(_HERE, "csrc", "*.h")) + \
+    deps = sources() + glob.glob(os.path.join(_HERE, "csrc", "*.h")) + glob.glob(os.path.join(_HERE, "csrc", "*.cuh")) + \
         glob.glob(os.path.join(_ROOT, "include", "*.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 

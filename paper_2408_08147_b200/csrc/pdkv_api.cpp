@@ -55,23 +55,7 @@ bool desc_ok(const pdkv_pool_desc *d)
     return true;
 }
 
-struct DeviceGuard {
-    int prev = -1;
-    bool changed = false;
-    cudaError_t err = cudaSuccess;
-    explicit DeviceGuard(int dev)
-    {
-        err = cudaGetDevice(&prev);
-        if (err == cudaSuccess && prev != dev) {
-            err = cudaSetDevice(dev);
-            changed = (err == cudaSuccess);
-        }
-    }
-    ~DeviceGuard()
-    {
-        if (changed) cudaSetDevice(prev);
-    }
-};
+using pdkv::DeviceGuard;
 
 }  // namespace
 
@@ -255,6 +239,7 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     cfg.unroll = (int)pdkv::tunables().unroll;
     cfg.threads = (int)pdkv::tunables().threads;
     cfg.ctas_per_sm = (int)pdkv::tunables().ctas_per_sm;
+    cfg.max_ctas = (int)pdkv::tunables().max_ctas;
     cfg.sm_count = pl->sm_count;
     cfg.variant = (int)pdkv::tunables().variant;
     cfg.check_bounds = pdkv::tunables().debug_bounds != 0;
@@ -775,6 +760,7 @@ int pdkv_tune(const char *key, int64_t value)
     const std::string k(key);
     if (k == "tile_bytes" && value >= 1 && value <= (1ll << 30)) t.tile_bytes = value;
     else if (k == "ctas_per_sm" && value >= 1 && value <= 32) t.ctas_per_sm = value;
+    else if (k == "max_ctas" && value >= 0 && value <= 65535) t.max_ctas = value;
     else if (k == "threads" && (value == 0 || (value >= 32 && value <= 1024 && value % 32 == 0))) t.threads = value;
     else if (k == "unroll" && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8)) t.unroll = value;
     else if (k == "vec32" && (value == 0 || value == 1)) t.vec32 = value;
@@ -796,6 +782,7 @@ int pdkv_tune_get(const char *key, int64_t *value)
     const std::string k(key);
     if (k == "tile_bytes") *value = t.tile_bytes;
     else if (k == "ctas_per_sm") *value = t.ctas_per_sm;
+    else if (k == "max_ctas") *value = t.max_ctas;
     else if (k == "threads") *value = t.threads;
     else if (k == "unroll") *value = t.unroll;
     else if (k == "vec32") *value = t.vec32;

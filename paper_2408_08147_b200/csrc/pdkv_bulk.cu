@@ -16,6 +16,7 @@
 //
 // Every wait is bounded: after kSpinLimit failed polls the warp records an
 // error word, drains its own stores and returns.
+#include "pdkv_device.cuh"
 #include "pdkv_internal.h"
 
 namespace pdkv {
@@ -66,9 +67,6 @@ __device__ __forceinline__ void bulk_s2g(void *gdst, const void *ssrc, uint32_t 
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-
-__device__ __forceinline__ uint32_t fast_div(uint32_t n, uint32_t m) { return m ? __umulhi(n, m) : n; }
-__device__ __forceinline__ uint32_t div_magic(uint32_t d) { return d == 1u ? 0u : 0xFFFFFFFFu / d + 1u; }
 
 struct Item {
     int64_t s_base, d_base;
@@ -258,6 +256,7 @@ cudaError_t launch_bulk(const CopyParams &p, const LaunchConfig &cfg, cudaStream
     if (occ < 1) return cudaErrorInvalidConfiguration;
     if (occ > cfg.ctas_per_sm) occ = cfg.ctas_per_sm;
     int64_t grid = (int64_t)cfg.sm_count * occ;
+    if (cfg.max_ctas > 0 && grid > cfg.max_ctas) grid = cfg.max_ctas;
     if (grid > n_work) grid = n_work;
     bulk_tiles_kernel<<<(unsigned)grid, 32, smem, stream>>>(p, stages, stage_bytes);
     return cudaGetLastError();

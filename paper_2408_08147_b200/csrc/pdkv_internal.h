@@ -49,6 +49,7 @@ struct LaunchConfig {
     int group_threads;  // threads per work item; the launcher rounds it to a divisor of `threads`
     int threads;
     int ctas_per_sm;
+    int max_ctas;    // 0: no cap; else the grid is limited to this many CTAs (leaves SMs to other kernels)
     int sm_count;
     int variant;
     int stages;              // bulk variant: shared-memory stages per CTA
@@ -63,9 +64,31 @@ cudaError_t launch_copy(const CopyParams &p, const LaunchConfig &cfg, cudaStream
 cudaError_t launch_bulk(const CopyParams &p, const LaunchConfig &cfg, cudaStream_t stream);
 bool bulk_supported(const LaunchConfig &cfg, int row_bytes);
 
+// Makes `dev` current for the lifetime of the object and restores the caller's device.
+struct DeviceGuard {
+    int prev = -1;
+    bool changed = false;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceGuard(int dev)
+    {
+        err = cudaGetDevice(&prev);
+        if (err == cudaSuccess && prev != dev) {
+            err = cudaSetDevice(dev);
+            changed = (err == cudaSuccess);
+        }
+    }
+    ~DeviceGuard()
+    {
+        if (changed) cudaSetDevice(prev);
+    }
+    DeviceGuard(const DeviceGuard &) = delete;
+    DeviceGuard &operator=(const DeviceGuard &) = delete;
+};
+
 struct Tunables {
     int64_t tile_bytes = 32768;
     int64_t ctas_per_sm = 2;
+    int64_t max_ctas = 0;
     int64_t threads = 0;   // 0: chosen with unroll, per class of copy
     int64_t unroll = 0;    // 0: chosen per class of copy
     int64_t vec32 = 1;

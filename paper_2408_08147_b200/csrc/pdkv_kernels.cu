@@ -8,6 +8,7 @@
 // rows, and the number of bytes each SM keeps in flight is a launch parameter
 // (threads x CTAs x unroll), because on B200 a copy runs fastest with about
 // 32-64 KiB of loads outstanding per SM, not with as many as fit.
+#include "pdkv_device.cuh"
 #include "pdkv_internal.h"
 
 namespace pdkv {
@@ -76,17 +77,6 @@ __device__ __forceinline__ bool in_bounds(int64_t off, int width, int64_t size)
 __device__ __forceinline__ void refuse(unsigned long long *status, int64_t off)
 {
     if (atomicCAS(status, 0ull, 1ull) == 0ull) status[1] = (unsigned long long)off;
-}
-
-// n / d through one multiply: m = floor(2^32 / d) + 1 (0 stands for d == 1).
-// Exact while n * d < 2^32, which the planner guarantees for every tile.
-__device__ __forceinline__ uint32_t fast_div(uint32_t n, uint32_t m)
-{
-    return m ? __umulhi(n, m) : n;
-}
-__device__ __forceinline__ uint32_t div_magic(uint32_t d)
-{
-    return d == 1u ? 0u : 0xFFFFFFFFu / d + 1u;  // for a power of two this is 2^32 / d, also exact
 }
 
 // Register copy: every thread issues U independent streaming loads, then
@@ -249,6 +239,7 @@ static cudaError_t launch_wu(const CopyParams &p, const LaunchConfig &cfg, cudaS
     q.group_threads = group;
     const int64_t per_cta = threads / group;
     int64_t grid = (int64_t)cfg.sm_count * occ;
+    if (cfg.max_ctas > 0 && grid > cfg.max_ctas) grid = cfg.max_ctas;
     if (grid * per_cta > n_work) grid = (n_work + per_cta - 1) / per_cta;
     kern<<<(unsigned)grid, threads, 0, stream>>>(q);
     return cudaGetLastError();

@@ -112,6 +112,7 @@ extern "C" int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
         cfg.unroll = t.unroll ? (int)t.unroll : 4;
         cfg.threads = t.threads ? (int)t.threads : 256;
         cfg.ctas_per_sm = (int)t.ctas_per_sm;
+        cfg.max_ctas = (int)t.max_ctas;
         cfg.sm_count = slot.sm_count;
         cfg.variant = 0;
         cfg.group_threads = cfg.threads;

@@ -41,20 +41,7 @@ Slot *find(pdkv_queue *q, int64_t ticket)
     return nullptr;
 }
 
-struct DevGuard {
-    int prev = -1;
-    bool changed = false;
-    cudaError_t err;
-    explicit DevGuard(int dev)
-    {
-        err = cudaGetDevice(&prev);
-        if (err == cudaSuccess && prev != dev) {
-            err = cudaSetDevice(dev);
-            changed = err == cudaSuccess;
-        }
-    }
-    ~DevGuard() { if (changed) cudaSetDevice(prev); }
-};
+using DevGuard = pdkv::DeviceGuard;
 
 }  // namespace
 
