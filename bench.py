@@ -37,9 +37,9 @@ KERNEL_SOURCE = os.path.join(ROOT, "paper_2408_08147_b200", "csrc", "pdkv_kernel
 # Captured on a 1/8-size case (4 of 32 requests; profiles/copy_tiles_kernel_config2_small_ncu_full.md)
 # and scaled by 8: traffic is proportional to the tokens moved (read 1.0738 GB + write 1.031 GB
 # per 2.1475 GB algorithmic).
-NCU_TRAFFIC: dict = {(2, "pack"): 8 * (1.073881e9 + 1.028534e9), (2, "unpack"): 8 * (1.073867e9 + 1.030490e9),
-                     (2, "fused"): 8 * (1.073860e9 + 1.029193e9)}
-NCU_KERNEL_SHA = "bb07cadbb5de7e6e"
+NCU_TRAFFIC: dict = {(2, "pack"): 8 * (1.073880e9 + 1.027572e9), (2, "unpack"): 8 * (1.073865e9 + 1.030411e9),
+                     (2, "fused"): 8 * (1.073906e9 + 1.029486e9)}
+NCU_KERNEL_SHA = "f142536d764dccc3"
 
 
 def log(*a):
