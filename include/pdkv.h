@@ -131,7 +131,10 @@ int pdkv_pool_destroy(pdkv_pool *pool);
  * transfer (Sec. 3.5).  `src` or `dst` may be NULL for a pack-only or
  * unpack-only plan (not both).  `skip_granule_tokens` must equal the decode
  * block size when `dst` is given; it is only free for pack-only plans (<= 0
- * selects it from `dst`).  One small host->device copy is enqueued on `stream`
+ * selects it from `dst`).  The two pools must not overlap in memory (there is
+ * no in-place re-blocking), nor may the contiguous buffer later passed to
+ * pack / unpack overlap the pool it is paired with: INVALID_ARG.  One small
+ * host->device copy is enqueued on `stream`
  * and the call waits for it; later calls on other streams are therefore safe.
  * Errors: INVALID_ARG, GEOMETRY, TABLE, CUDA, NOMEM; *out is NULL on error. */
 int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst,

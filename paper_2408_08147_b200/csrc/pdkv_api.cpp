@@ -279,6 +279,13 @@ bool layers_ok(const pdkv_plan *pl, int l0, int l1) { return l0 >= 0 && l0 <= l1
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The kernels read one side while writing the other, with no ordering between tiles.
+bool ranges_overlap(const void *a, size_t a_bytes, const void *b, size_t b_bytes)
+{
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a_bytes && b_bytes && a0 < b0 + b_bytes && b0 < a0 + a_bytes;
+}
+
 }  // namespace
 
 namespace pdkv {
@@ -361,6 +368,8 @@ int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip_gr
             src->d.head_dim != dst->d.head_dim || src->d.elem_bytes != dst->d.elem_bytes)
             return PDKV_ERR_GEOMETRY;
         if (src->device != dst->device) return PDKV_ERR_INVALID_ARG;
+        if (ranges_overlap(src->base, pdkv_pool_bytes(&src->d), dst->base, pdkv_pool_bytes(&dst->d)))
+            return PDKV_ERR_INVALID_ARG;   // in-place re-blocking is not supported
     }
     int32_t G = skip_granule_tokens;
     if (dst) {
@@ -590,6 +599,8 @@ int pdkv_pack(const pdkv_plan *plan, void *buf, size_t buf_bytes, int l0, int l1
     if (!plan->dev_mem) return PDKV_ERR_INVALID_ARG;  // host-only plan
     if (plan->payload_bytes == 0 || l0 == l1) return PDKV_OK;
     if (!buf || !aligned16(buf)) return PDKV_ERR_INVALID_ARG;
+    if (ranges_overlap(buf, plan->payload_bytes, plan->src.base, pdkv_pool_bytes(&plan->src.d)))
+        return PDKV_ERR_INVALID_ARG;
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
     return launch_op(plan, PDKV_OP_PACK, pool_side(plan->src, plan->row_bytes, plan->hrow_bytes),
@@ -604,6 +615,8 @@ int pdkv_unpack(const pdkv_plan *plan, const void *buf, size_t buf_bytes, int l0
     if (!plan->dev_mem) return PDKV_ERR_INVALID_ARG;  // host-only plan
     if (plan->tiles[PDKV_OP_UNPACK].empty() || l0 == l1) return PDKV_OK;
     if (plan->payload_bytes && (!buf || !aligned16(buf))) return PDKV_ERR_INVALID_ARG;
+    if (ranges_overlap(buf, plan->payload_bytes, plan->dst.base, pdkv_pool_bytes(&plan->dst.d)))
+        return PDKV_ERR_INVALID_ARG;
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
     return launch_op(plan, PDKV_OP_UNPACK, buffer_side(buf, buf_bytes, plan->row_bytes, plan->hrow_bytes),

@@ -105,6 +105,12 @@ def test_plan_validation_errors():
     with pytest.raises(B.PdkvError) as e:
         _plan(w, ps, other)
     assert e.value.status == B.PDKV_ERR_GEOMETRY
+    # overlapping pools (in-place re-blocking) are refused
+    near = B.pdkv_pool_create(B.desc_of(w.dst), FAKE_BASE + 4096, w.dst.num_bytes(), 0)
+    with pytest.raises(B.PdkvError) as e:
+        _plan(w, ps, near)
+    assert e.value.status == B.PDKV_ERR_INVALID_ARG
+    B.pdkv_pool_destroy(near)
     # skip granule must be the decode block
     with pytest.raises(B.PdkvError) as e:
         B.pdkv_plan_create(ps, pd, 16, b.seq_len, b.src_tbl_off, b.src_tbl, b.dst_tbl_off, b.dst_tbl)
@@ -132,6 +138,9 @@ def test_launch_argument_errors_and_dry_run_refusal():
     with pytest.raises(B.PdkvError) as e:
         B.pdkv_pack(plan, FAKE_BASE, total - 1, 0, 2)
     assert e.value.status == B.PDKV_ERR_BUFFER_TOO_SMALL
+    with pytest.raises(B.PdkvError) as e:               # buffer inside the decode pool
+        B.pdkv_unpack(plan, FAKE_BASE + (1 << 40) + 256, total, 0, 2)
+    assert e.value.status == B.PDKV_ERR_INVALID_ARG
     # a dry-run plan owns no device arrays: launching is refused, not attempted
     for fn, args in [(B.pdkv_pack, (plan, FAKE_BASE, total, 0, 2)),
                      (B.pdkv_transfer, (plan, 0, 2)), (B.pdkv_transfer_blockwise, (plan,)),
