@@ -273,7 +273,16 @@ def cpu_baseline(w, src_t, budget_s=20.0):
     oracle_step(O, sub, src_np, dst_np, buf_np, threads)
     dt = time.perf_counter() - t0
     nbytes = step_bytes_of(sub)
+    # the same checker on one request with one thread, for a per-core figure
+    one, one_ids, _ = W.compact_subproblem(w, [0])
+    one_src = W.gather_blocks(src_t.view(__import__("torch").int16), w.src, one_ids).cpu().numpy().view(np.uint16)
+    one_dst = W.sentinel_pool_numpy(one.dst)
+    one_buf = np.zeros(O.buffer_elems(one.batch, one.dst.block_tokens, one.src), np.uint16)
+    t1 = time.perf_counter()
+    oracle_step(O, one, one_src, one_dst, one_buf, 1)
+    dt1 = time.perf_counter() - t1
     return {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "single_thread_value": step_bytes_of(one) / dt1 / 1e9,
             "sample": f"first {n} of {w.batch.n_req} requests ({int(sub.batch.seq_len.sum())} tokens, "
                       f"all layers), one pack+unpack+fused pass, {dt:.2f} s wall",
             "host_cpus": cores}
@@ -720,7 +729,7 @@ def parse():
     ap.add_argument("--layouts", default="", help="two letters, e.g. AB: prefill block-major, decode layer-major")
     ap.add_argument("--tune", nargs=2, action="append", metavar=("KEY", "VALUE"))
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--e2e-groups", type=int, default=8, help="request groups pipelined over three streams in the e2e leg")
+    ap.add_argument("--e2e-groups", type=int, default=16, help="request groups pipelined over three streams in the e2e leg")
     ap.add_argument("--no-extras", action="store_true", help="skip baseline, e2e and CPU legs")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
