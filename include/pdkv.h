@@ -306,8 +306,9 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream);
  *                    budget of the chosen variant allows; 0 = automatic (default)
  *   "unroll"         independent accesses in flight per thread: 1, 2, 4, 8;
  *                    0 = automatic (default).  Automatic means 512 threads x 1
- *                    access for flat copies (token-major on both sides) and
- *                    256 threads x 4 for copies with a head-major side
+ *                    access for flat copies (token-major on both sides) and for
+ *                    batches of small tiles, 256 threads x 4 for full-tile
+ *                    copies with a head-major side
  *   "group_threads"  threads that cooperate on one work item (a CTA hosts
  *                    threads / group_threads independent groups); 0 = automatic
  *                    (default): sized so that the plan's mean tile is covered in

@@ -243,20 +243,22 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     cfg.sm_count = pl->sm_count;
     cfg.variant = (int)pdkv::tunables().variant;
     cfg.check_bounds = pdkv::tunables().debug_bounds != 0;
-    {   // automatic launch shape, measured best per class of copy on B200: a flat copy
-        // (token-major on both sides) runs 512 threads with one access in flight each, a
-        // row-permuting or head-major copy 256 threads with four, i.e. one 32 KiB tile per pass
+    {   // Automatic launch shape, measured best per class of copy on B200.  Full tiles
+        // (about 32 KiB): a flat copy (token-major on both sides) runs 512 threads with
+        // one access in flight each, i.e. two passes per tile; a copy with a head-major
+        // side runs 256 threads with four, i.e. one pass per tile.  Batches of small
+        // tiles (few KV heads, short blocks): groups of threads that cover a tile in two
+        // passes of one access each, 32 threads at least.
         const int64_t hrow = pl->hrow_bytes, row = pl->row_bytes;
         const bool flat = src.head_stride == row && src.tok_stride == hrow && dst.head_stride == row &&
                           dst.tok_stride == hrow;
-        if (cfg.unroll == 0) cfg.unroll = flat ? 1 : 4;
-        if (cfg.threads == 0) cfg.threads = flat ? 512 : 256;
-        // threads per work item: a flat tile is covered in two passes, any other in one, so
-        // that batches of small tiles (few KV heads, small blocks) still fill the CTA
+        const bool small = pl->mean_tile_bytes[op] < 24 * 1024;
+        if (cfg.unroll == 0) cfg.unroll = (flat || small) ? 1 : 4;
+        if (cfg.threads == 0) cfg.threads = (flat || small) ? 512 : 256;
         cfg.group_threads = (int)pdkv::tunables().group_threads;
         if (cfg.group_threads == 0) {
             const int64_t vecs = std::max<int64_t>(1, pl->mean_tile_bytes[op] / cfg.vec_bytes);
-            const int64_t want = vecs / (flat ? 2 : cfg.unroll);
+            const int64_t want = vecs / ((flat || small) ? 2 : cfg.unroll);
             int g = 32;
             while (g < want && g < cfg.threads) g *= 2;
             cfg.group_threads = g;
