@@ -617,7 +617,11 @@ def overlap_arm(args):
              ("register copy on at most 32 SMs", {"variant": 0, "ctas_per_sm": 1, "threads": 1024, "unroll": 1,
                                                   "max_ctas": 32}),
              ("bulk copy (TMA), 8 KiB tiles x 2 stages x 8 CTAs/SM",
-              {"variant": 1, "tile_bytes": 8192, "stages": 2, "ctas_per_sm": 8})]
+              {"variant": 1, "tile_bytes": 8192, "stages": 2, "ctas_per_sm": 8}),
+             ("bulk copy with tiled TMA loads, 16 KiB tiles x 4 stages x 3 CTAs/SM",
+              {"variant": 2, "tile_bytes": 16384, "stages": 4, "ctas_per_sm": 3}),
+             ("bulk copy with tiled TMA loads, 16 KiB tiles x 2 stages x 2 CTAs/SM",
+              {"variant": 2, "tile_bytes": 16384, "stages": 2, "ctas_per_sm": 2})]
     defaults = {k: B.pdkv_tune_get(k) for k in ("variant", "ctas_per_sm", "threads", "unroll", "tile_bytes", "stages",
                                                 "max_ctas")}
     t_compute = timed(compute_only, args.steps)

@@ -242,6 +242,7 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     cfg.max_ctas = (int)pdkv::tunables().max_ctas;
     cfg.sm_count = pl->sm_count;
     cfg.variant = (int)pdkv::tunables().variant;
+    cfg.elem_bytes = pl->E;
     cfg.check_bounds = pdkv::tunables().debug_bounds != 0;
     {   // Automatic launch shape, measured best per class of copy on B200.  Full tiles
         // (about 32 KiB): a flat copy (token-major on both sides) runs 512 threads with
@@ -267,7 +268,7 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     cfg.stages = (int)pdkv::tunables().stages;
     cfg.max_tile_bytes = pl->max_tile_bytes;
     cudaError_t e;
-    if (cfg.variant == 1 && pdkv::bulk_supported(cfg, p.row_bytes)) {
+    if (cfg.variant >= 1 && pdkv::bulk_supported(cfg, p.row_bytes)) {
         cfg.vec_bytes = 16;
         e = pdkv::launch_bulk(p, cfg, stream);
     } else {
@@ -783,7 +784,7 @@ int pdkv_tune(const char *key, int64_t value)
     else if (k == "chunked" && (value == 0 || value == 1)) t.chunked = value;
     else if (k == "group_threads" && (value == 0 || (value >= 32 && value <= 1024 && value % 32 == 0))) t.group_threads = value;
     else if (k == "debug_bounds" && (value == 0 || value == 1)) t.debug_bounds = value;
-    else if (k == "variant" && value >= 0 && value <= 1) t.variant = value;
+    else if (k == "variant" && value >= 0 && value <= 2) t.variant = value;
     else if (k == "stages" && value >= 2 && value <= 16) t.stages = value;
     else if (k == "dry_run" && (value == 0 || value == 1)) t.dry_run = value;
     else return PDKV_ERR_INVALID_ARG;

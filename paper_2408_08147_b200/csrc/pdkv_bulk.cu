@@ -14,8 +14,22 @@
 // or the contiguous buffer) the stage is [token][head][row] and the store is a
 // single bulk copy.
 //
+// With "variant" 2 the transpose of a token-major source into a head-major
+// destination is done by the TMA unit itself: the source side (a block-major
+// pool or the contiguous buffer, both a dense [token row][head][dim] array) is
+// described by a 3-D tensor map, and one tiled load with the box
+// (dim = D, head = 1, tokens = T) fetches the T strided rows of one head into a
+// dense [T][D] piece of the stage -- H loads per tile instead of one per row.
+// The innermost coordinate of every load is 0 (16-byte rule), stage pieces are
+// 128-byte aligned, and a box may over-read past a ragged tile (reads only;
+// out-of-range rows are zero-filled by the hardware and never stored).
+//
 // Every wait is bounded: after kSpinLimit failed polls the warp records an
 // error word, drains its own stores and returns.
+#include <cstring>
+
+#include <cuda.h>
+
 #include "pdkv_device.cuh"
 #include "pdkv_internal.h"
 
@@ -58,6 +72,15 @@ __device__ __forceinline__ void bulk_g2s(void *sdst, const void *gsrc, uint32_t 
                  "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
+// Tiled 3-D load: box (D, 1, T) at coordinates (0, head, token row).
+__device__ __forceinline__ void tensor_g2s(void *sdst, const CUtensorMap *map, int head, int tok_row, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+            smem_u32(sdst)),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(head), "r"(tok_row), "r"(smem_u32(bar))
+        : "memory");
+}
 __device__ __forceinline__ void bulk_s2g(void *gdst, const void *ssrc, uint32_t bytes)
 {
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(ssrc)),
@@ -76,8 +99,12 @@ struct Item {
 
 }  // namespace
 
-__global__ void __launch_bounds__(32) bulk_tiles_kernel(const CopyParams p, const int stages, const uint32_t stage_bytes)
+__global__ void __launch_bounds__(32)
+bulk_tiles_kernel(const CopyParams p, const int stages, const uint32_t stage_bytes,
+                  const __grid_constant__ CUtensorMap src_map, const int map_tokens)
 {
+    // map_tokens > 0: src_map describes the source as [token row][head][dim] and its box holds
+    // map_tokens tokens of one head; used for token-major -> head-major tiles only
     extern __shared__ __align__(128) unsigned char smem[];
     uint64_t *full = reinterpret_cast<uint64_t *>(smem);
     unsigned char *data = smem + kBarrierBytes;
@@ -90,6 +117,8 @@ __global__ void __launch_bounds__(32) bulk_tiles_kernel(const CopyParams p, cons
     const bool src_flat = p.src.head_stride == p.row_bytes && p.src.tok_stride == hrow;
     const bool dst_flat = p.dst.head_stride == p.row_bytes && p.dst.tok_stride == hrow;
     const uint32_t m_H = div_magic(H);
+    const bool tiled = map_tokens > 0 && src_tok_major && !dst_tok_major;
+    const uint32_t piece = tiled ? (uint32_t)map_tokens * row : 0;   // stage bytes per head
 
     if (lane == 0) {
         for (int i = 0; i < stages; ++i) mbar_init(full + i, 1);
@@ -140,6 +169,13 @@ __global__ void __launch_bounds__(32) bulk_tiles_kernel(const CopyParams p, cons
         const uint32_t bytes = it.ntok * H * row;
         if (it.zero) {                      // nothing to fetch; the store side writes zeros itself
             if (lane == 0) mbar_arrive(bar);
+            return;
+        }
+        if (tiled) {                        // H boxes of map_tokens x row bytes, whatever ntok is
+            if (lane == 0) mbar_arrive_expect(bar, H * piece);
+            __syncwarp();
+            const int tok_row = (int)(it.s_base / hrow);
+            for (uint32_t hd = lane; hd < H; hd += 32) tensor_g2s(st + (size_t)hd * piece, &src_map, (int)hd, tok_row, bar);
             return;
         }
         if (lane == 0) mbar_arrive_expect(bar, bytes);
@@ -201,7 +237,8 @@ __global__ void __launch_bounds__(32) bulk_tiles_kernel(const CopyParams p, cons
                 bulk_s2g(dst + tk * p.dst.tok_stride, st + (size_t)tk * H * row, H * row);
         } else {                            // head-major: one run per head
             const uint32_t run = it.ntok * row;
-            for (uint32_t hd = lane; hd < H; hd += 32) bulk_s2g(dst + hd * p.dst.head_stride, st + (size_t)hd * run, run);
+            const uint32_t pitch = tiled ? piece : run;   // tiled stages keep map_tokens rows per head
+            for (uint32_t hd = lane; hd < H; hd += 32) bulk_s2g(dst + hd * p.dst.head_stride, st + (size_t)hd * pitch, run);
         }
         bulk_commit();
     };
@@ -241,11 +278,67 @@ __global__ void __launch_bounds__(32) bulk_tiles_kernel(const CopyParams p, cons
     bulk_wait_all();
 }
 
+namespace {
+
+using EncodeTiled = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                 const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiled encode_tiled()
+{
+    static EncodeTiled fn = [] {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            sym = nullptr;
+        return reinterpret_cast<EncodeTiled>(sym);
+    }();
+    return fn;
+}
+
+// Tensor map of a token-major side viewed as [token rows][H][D]; box = (D, 1, tokens).
+// Returns false when the geometry does not meet the TMA rules (the caller then
+// uses per-row bulk copies).
+bool make_source_map(const CopyParams &p, int elem_bytes, int tokens, CUtensorMap *out)
+{
+    const int64_t row = p.row_bytes, hrow = (int64_t)p.H * row;
+    if (elem_bytes != 1 && elem_bytes != 2 && elem_bytes != 4 && elem_bytes != 8) return false;
+    const int64_t D = row / elem_bytes;
+    const int64_t rows = p.src.size / hrow;
+    if (!encode_tiled() || D < 1 || D > 256 || tokens < 1 || tokens > 256 || row % 16 || rows < 1 ||
+        rows > 0x7FFFFFFFll || ((int64_t)tokens * row) % 128 || (reinterpret_cast<uintptr_t>(p.src.base) & 15u) ||
+        hrow >= (1ll << 40))
+        return false;
+    const CUtensorMapDataType dt = elem_bytes == 1   ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                   : elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16
+                                   : elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT32
+                                                     : CU_TENSOR_MAP_DATA_TYPE_UINT64;
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)p.H, (cuuint64_t)rows};
+    const cuuint64_t strides[2] = {(cuuint64_t)row, (cuuint64_t)hrow};   // bytes, dimensions 1 and 2
+    const cuuint32_t box[3] = {(cuuint32_t)D, 1u, (cuuint32_t)tokens};
+    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    return encode_tiled()(out, dt, 3, p.src.base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
 cudaError_t launch_bulk(const CopyParams &p, const LaunchConfig &cfg, cudaStream_t stream)
 {
     const int64_t n_work = (int64_t)p.n_tiles * p.n_lc;
     if (n_work <= 0) return cudaSuccess;
     const uint32_t stage_bytes = (uint32_t)((cfg.max_tile_bytes + 127) / 128 * 128);
+    CUtensorMap map;
+    std::memset(&map, 0, sizeof(map));
+    int map_tokens = 0;
+    const bool src_tok_major = p.src.tok_stride >= p.src.head_stride;
+    const bool dst_tok_major = p.dst.tok_stride >= p.dst.head_stride;
+    if (cfg.variant == 2 && src_tok_major && !dst_tok_major) {
+        const int tokens = (int)(cfg.max_tile_bytes / ((int64_t)p.H * p.row_bytes));
+        if (make_source_map(p, cfg.elem_bytes, tokens, &map)) map_tokens = tokens;
+    }
     const int stages = cfg.stages;
     const size_t smem = kBarrierBytes + (size_t)stages * stage_bytes;
     cudaError_t e = cudaFuncSetAttribute(bulk_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -258,7 +351,7 @@ cudaError_t launch_bulk(const CopyParams &p, const LaunchConfig &cfg, cudaStream
     int64_t grid = (int64_t)cfg.sm_count * occ;
     if (cfg.max_ctas > 0 && grid > cfg.max_ctas) grid = cfg.max_ctas;
     if (grid > n_work) grid = n_work;
-    bulk_tiles_kernel<<<(unsigned)grid, 32, smem, stream>>>(p, stages, stage_bytes);
+    bulk_tiles_kernel<<<(unsigned)grid, 32, smem, stream>>>(p, stages, stage_bytes, map, map_tokens);
     return cudaGetLastError();
 }
 

@@ -51,7 +51,8 @@ struct LaunchConfig {
     int ctas_per_sm;
     int max_ctas;    // 0: no cap; else the grid is limited to this many CTAs (leaves SMs to other kernels)
     int sm_count;
-    int variant;
+    int variant;             // 0 register copy, 1 bulk copies, 2 bulk copies with tiled TMA loads
+    int elem_bytes;          // element size, for the tensor map's data type
     int stages;              // bulk variant: shared-memory stages per CTA
     int64_t max_tile_bytes;  // bulk variant: largest tile of the launch
     bool check_bounds;

@@ -115,6 +115,7 @@ extern "C" int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
         cfg.max_ctas = (int)t.max_ctas;
         cfg.sm_count = slot.sm_count;
         cfg.variant = 0;
+        cfg.elem_bytes = 0;
         cfg.group_threads = cfg.threads;
         cfg.stages = 0;
         cfg.max_tile_bytes = 0;

@@ -124,11 +124,14 @@ def test_tile_size_and_work_order_do_not_change_the_result(oracle, tile_bytes, l
         B.pdkv_tune("lc_fastest", 0)
 
 
+@pytest.mark.parametrize("variant", [1, 2])
 @pytest.mark.parametrize("stages,tile_bytes,chunked", [(2, 16384, 0), (3, 65536, 0), (4, 32768, 1)])
-def test_bulk_copy_variant(oracle, stages, tile_bytes, chunked):
-    """Variant 1 (TMA bulk copies through a shared-memory ring) must produce the
-    same bytes: flat, head-run and transposing tiles, zero-fill tiles, skip masks."""
-    B.pdkv_tune("variant", 1)
+def test_bulk_copy_variant(oracle, variant, stages, tile_bytes, chunked):
+    """Variants 1 and 2 (TMA bulk copies through a shared-memory ring; 2 adds tiled
+    tensor-map loads for the token-major -> head-major transpose) must produce the
+    same bytes: flat, head-run and transposing tiles, ragged and zero-fill tiles,
+    skip masks."""
+    B.pdkv_tune("variant", variant)
     B.pdkv_tune("stages", stages)
     B.pdkv_tune("tile_bytes", tile_bytes)
     B.pdkv_tune("chunked", chunked)
