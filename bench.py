@@ -682,7 +682,7 @@ def retrieval_arm(args):
     torch.cuda.synchronize()
     ps = B.pdkv_pool_create(B.desc_of(w.src), src_t.data_ptr(), src_t.numel(), 0)
     pd = B.pdkv_pool_create(B.desc_of(w.dst), dst_t.data_ptr(), dst_t.numel(), 0)
-    n_groups = max(1, min(args.e2e_groups, w.batch.n_req))
+    n_groups = max(1, min(args.retrieval_groups, w.batch.n_req))
     cuts = [round(i * w.batch.n_req / n_groups) for i in range(n_groups + 1)]
     groups = [W.slice_batch(w.batch, cuts[i], cuts[i + 1]) for i in range(n_groups)]
     out = {"mode": "retrieval", "config": {"workload": workload_name(w), "groups": n_groups}, "capacities": {}}
@@ -739,6 +739,7 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--overlap", action="store_true", help="per-layer transfer overlapped with a compute stand-in")
     ap.add_argument("--retrieval", action="store_true", help="request groups through the asynchronous retrieval queue")
+    ap.add_argument("--retrieval-groups", type=int, default=8)
     ap.add_argument("--gemm-n", type=int, default=4096)
     ap.add_argument("--side-priority", type=int, default=1, help="1: transfer stream has high priority")
     ap.add_argument("--no-blockwise", action="store_true")
