@@ -147,6 +147,19 @@ def barrier():
         dist.barrier()
 
 
+def all_ranks_agree(flag: bool, device=None) -> bool:
+    """True only if every rank passed True (a collective decision, so that all ranks
+    take the same branch around later barriers)."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()):
+        return bool(flag)
+    t = torch.tensor([1 if flag else 0], dtype=torch.int32, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MIN)
+    return bool(t.item())
+
+
 def reduce_step_time(ms_local: float, units_local: float, device=None):
     """Max of the per-rank times and sum of the per-rank units, on every rank."""
     import torch
@@ -499,12 +512,21 @@ def e2e_leg(args, w, src_t, dst_t, buf_t, stream, step_bytes, torch, B, Transfer
         pass
     _, _, world = dist_env()
     need = (src_t.numel() + dst_t.numel()) * world      # every rank on this node pins its own images
-    if free_host is not None and need > 0.5 * free_host:
+    fits = not (free_host is not None and need > 0.5 * free_host)
+    fits = all_ranks_agree(fits, dev)     # one rank skipping alone would leave the others in a barrier
+    if not fits:
         return {"value": None, "unit": UNIT,
                 "skipped": f"needs {need >> 30} GiB of pinned host memory across {world} ranks, "
-                           f"{free_host >> 30} GiB available"}
-    h_src = torch.empty(src_t.numel(), dtype=torch.uint8, pin_memory=True)
-    h_dst = torch.empty(dst_t.numel(), dtype=torch.uint8, pin_memory=True)
+                           f"{(free_host or 0) >> 30} GiB available"}
+    try:
+        h_src = torch.empty(src_t.numel(), dtype=torch.uint8, pin_memory=True)
+        h_dst = torch.empty(dst_t.numel(), dtype=torch.uint8, pin_memory=True)
+        pinned = True
+    except RuntimeError:
+        h_src = h_dst = None
+        pinned = False
+    if not all_ranks_agree(pinned, dev):
+        return {"value": None, "unit": UNIT, "skipped": "pinned host allocation failed on a rank"}
     h_src.copy_(src_t)
     steps = max(1, min(args.e2e_steps, args.steps))
     up_down = [0, 0]

@@ -27,8 +27,10 @@ def _worker(rank, world, port, q):
     r, w = bench.dist_init("gloo")
     bench.barrier()
     ms, units = bench.reduce_step_time(10.0 + 5.0 * rank, 100.0 * (rank + 1))
+    agree_all = bench.all_ranks_agree(True)
+    agree_one = bench.all_ranks_agree(rank == 0)      # rank 1 objects: nobody proceeds
     bench.barrier()
-    q.put((r, w, ms, units))
+    q.put((r, w, ms, units, agree_all, agree_one))
     import torch.distributed as dist
 
     dist.destroy_process_group()
@@ -48,8 +50,9 @@ def test_time_is_max_and_units_are_summed_over_ranks():
         p.join(timeout=60)
         assert p.exitcode == 0
     assert [g[0] for g in got] == [0, 1]
-    for _, world, ms, units in got:
+    for _, world, ms, units, agree_all, agree_one in got:
         assert world == 2 and ms == 15.0 and units == 300.0
+        assert agree_all is True and agree_one is False
 
 
 def test_single_process_needs_no_process_group():
@@ -57,6 +60,7 @@ def test_single_process_needs_no_process_group():
     import bench
 
     assert bench.reduce_step_time(3.0, 7.0) == (3.0, 7.0)
+    assert bench.all_ranks_agree(True) and not bench.all_ranks_agree(False)
     bench.barrier()
 
 

@@ -296,3 +296,13 @@ def test_block_bytes_count_referenced_and_written_blocks():
     assert len(src_ids) < w.src.num_blocks            # resident prefixes are not uploaded
     B.pdkv_plan_destroy(plan)
     B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    """There is no CPU fallback: without the built library the binding raises."""
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "libpdkv_absent.so"))
+    with pytest.raises(ImportError):
+        B.lib()
+    with pytest.raises(ImportError):
+        B.pdkv_pool_bytes(B.make_desc(0, 1, 1, 8, 2, 4, 2))
