@@ -319,6 +319,8 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream);
  *   "chunked"        1: each CTA takes one contiguous run of work items instead
  *                    of every gridDim-th one (default 0)
  *   "debug_bounds"   1: kernels range-check every access and skip bad ones
+ *   "debug_shrink"   with "debug_bounds": pretend each side is N bytes shorter, so
+ *                    that the refusal path can be exercised on valid memory
  *   "variant"        0: register copy (default); 1: bulk async copies (TMA) through
  *                    shared memory, one warp per CTA; used when rows are multiples
  *                    of 16 bytes and a tile fits a stage, else variant 0 runs;

@@ -221,6 +221,10 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     pdkv::CopyParams p;
     p.src = src;
     p.dst = dst;
+    if (pdkv::tunables().debug_bounds && pdkv::tunables().debug_shrink > 0) {
+        p.src.size = std::max<int64_t>(0, p.src.size - pdkv::tunables().debug_shrink);
+        p.dst.size = std::max<int64_t>(0, p.dst.size - pdkv::tunables().debug_shrink);
+    }
     p.tiles = pl->dev_tiles[op];
     p.tile_begin = tile_begin;
     p.n_tiles = n_tiles;
@@ -784,6 +788,7 @@ int pdkv_tune(const char *key, int64_t value)
     else if (k == "chunked" && (value == 0 || value == 1)) t.chunked = value;
     else if (k == "group_threads" && (value == 0 || (value >= 32 && value <= 1024 && value % 32 == 0))) t.group_threads = value;
     else if (k == "debug_bounds" && (value == 0 || value == 1)) t.debug_bounds = value;
+    else if (k == "debug_shrink" && value >= 0) t.debug_shrink = value;
     else if (k == "variant" && value >= 0 && value <= 2) t.variant = value;
     else if (k == "stages" && value >= 2 && value <= 16) t.stages = value;
     else if (k == "dry_run" && (value == 0 || value == 1)) t.dry_run = value;
@@ -806,6 +811,7 @@ int pdkv_tune_get(const char *key, int64_t *value)
     else if (k == "chunked") *value = t.chunked;
     else if (k == "group_threads") *value = t.group_threads;
     else if (k == "debug_bounds") *value = t.debug_bounds;
+    else if (k == "debug_shrink") *value = t.debug_shrink;
     else if (k == "variant") *value = t.variant;
     else if (k == "stages") *value = t.stages;
     else if (k == "dry_run") *value = t.dry_run;

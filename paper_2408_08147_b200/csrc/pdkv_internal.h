@@ -97,6 +97,7 @@ struct Tunables {
     int64_t group_threads = 0;   // 0: sized from the plan's mean tile
     int64_t chunked = 0;
     int64_t debug_bounds = 0;
+    int64_t debug_shrink = 0;   // with debug_bounds: treat the last N bytes of each side as out of range
     int64_t variant = 0;
     int64_t stages = 3;
     int64_t dry_run = 0;

@@ -324,3 +324,45 @@ def test_per_layer_calls_replayed_from_a_cuda_graph(oracle):
         graph.replay()
         torch.cuda.synchronize()
         assert np.array_equal(host(dst_t), want)
+
+
+def test_bounds_checked_kernels_refuse_and_skip(oracle):
+    """With the range check on and both sides declared 4 KiB shorter than they are,
+    accesses into the last 4 KiB are refused: they are skipped (the sentinel
+    survives), everything else is copied, and the plan reports the refusal."""
+    from paper_2408_08147_b200.session import TransferSession
+
+    w = W.make_config(2, num_layers=2, n_req=2, max_len=256)      # block-major both sides, every block used
+    src = W.fill_pool_numpy(w.src, w.seed)
+    sent = W.sentinel_pool_numpy(w.dst)
+    want = sent.copy()
+    oracle.transfer(w.src, src, w.dst, want, w.batch)
+    src_t, dst_t = dev(src), dev(sent)
+    torch.cuda.synchronize()
+    B.pdkv_tune("debug_bounds", 1)
+    B.pdkv_tune("debug_shrink", 4096)
+    try:
+        with TransferSession(w.src, src_t, w.dst, dst_t, w.batch) as s:
+            s.transfer()
+            with pytest.raises(B.PdkvError) as e:
+                s.status()
+            assert e.value.status == B.PDKV_ERR_DEVICE_BOUNDS and "refused" in str(e.value)
+        # Both pools are [block][layer][K/V][token][head][dim] with 2 KiB per token, so the last
+        # 4 KiB of a pool are tokens 126..127 of its last block's last (layer, V) strip.  Refused:
+        # the writes into the decode pool's tail, and the reads of the prefill pool's tail (whose
+        # destination is found through the tables; same block size on both sides).
+        expect = want.copy().reshape(w.dst.shape())
+        L, NB = w.dst.num_layers, w.dst.num_blocks
+        expect[NB - 1, L - 1, 1, 126:128] = SENT
+        pos = int(np.flatnonzero(w.batch.src_tbl == w.src.num_blocks - 1)[0])
+        expect[int(w.batch.dst_tbl[pos]), L - 1, 1, 126:128] = SENT
+        assert np.array_equal(host(dst_t), expect.reshape(-1))
+        # a clean run on the same plan data clears nothing by itself: a fresh plan reports OK
+        B.pdkv_tune("debug_shrink", 0)
+        dst_t.copy_(dev(sent)); torch.cuda.synchronize()
+        with TransferSession(w.src, src_t, w.dst, dst_t, w.batch) as s:
+            s.transfer(); s.status()
+        assert np.array_equal(host(dst_t), want)
+    finally:
+        B.pdkv_tune("debug_bounds", 0)
+        B.pdkv_tune("debug_shrink", 0)
