@@ -140,6 +140,8 @@ int pdkv_pool_destroy(pdkv_pool *pool);
 int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst,
                      int32_t skip_granule_tokens, const pdkv_batch_desc *batch,
                      void *stream, pdkv_plan **out);
+/* Frees the plan and its device arrays.  Call it once the work enqueued with
+ * the plan has completed (its kernels read the tile lists). */
 int pdkv_plan_destroy(pdkv_plan *plan);
 
 /* Size of the contiguous buffer in bytes and, optionally, the host array of
