@@ -366,3 +366,42 @@ def test_bounds_checked_kernels_refuse_and_skip(oracle):
     finally:
         B.pdkv_tune("debug_bounds", 0)
         B.pdkv_tune("debug_shrink", 0)
+
+
+@pytest.mark.parametrize("idx,kw", [(3, dict(num_layers=2, n_req=8, max_len=900)), (5, dict(num_layers=2, n_req=30))])
+def test_sender_only_and_receiver_only_plans(oracle, idx, kw):
+    """The two halves as separate devices would run them (Sec. 3.5): the sender
+    holds only the prefill pool and a pack-only plan, the receiver only the decode
+    pool and an unpack-only plan; the buffer travels as one copy in between.  (Here
+    both halves run on the same GPU; the buffer copy stands in for the link.)"""
+    from paper_2408_08147_b200.session import TransferSession
+
+    w = W.make_config(idx, **kw)
+    G = w.dst.block_tokens
+    src = W.fill_pool_numpy(w.src, w.seed)
+    sent = W.sentinel_pool_numpy(w.dst)
+    want = sent.copy()
+    oracle.transfer(w.src, src, w.dst, want, w.batch)
+    src_t, dst_t = dev(src), dev(sent)
+    torch.cuda.synchronize()
+    sender = TransferSession(w.src, src_t, None, None, w.batch, skip_granule_tokens=G)
+    receiver = TransferSession(None, None, w.dst, dst_t, w.batch)
+    try:
+        assert sender.buffer_bytes == receiver.buffer_bytes == oracle.buffer_elems(w.batch, G, w.src) * 2
+        assert np.array_equal(sender.request_offsets, receiver.request_offsets)
+        send_buf = torch.zeros(sender.buffer_bytes, dtype=torch.uint8, device="cuda")
+        recv_buf = torch.empty_like(send_buf)
+        L = w.src.num_layers
+        for l in range(L):                                  # per-layer trigger: offset and length per layer
+            sender.pack(send_buf, (l, l + 1))
+        recv_buf.copy_(send_buf)                            # "transfer all the data as a whole"
+        receiver.unpack(recv_buf)
+        torch.cuda.synchronize()
+        assert np.array_equal(host(dst_t), want)
+        with pytest.raises(B.PdkvError):
+            sender.transfer()
+        with pytest.raises(B.PdkvError):
+            receiver.pack(send_buf)
+    finally:
+        sender.close()
+        receiver.close()
