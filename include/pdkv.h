@@ -326,10 +326,11 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream);
  *   "variant"        0: register copy (default); 1: bulk async copies (TMA) through
  *                    shared memory, one warp per CTA; used when rows are multiples
  *                    of 16 bytes and a tile fits a stage, else variant 0 runs;
- *                    2: as 1, and tiles going from a token-major source to a
- *                    head-major pool are fetched with tiled TMA loads through a
- *                    tensor map of the source (one load per head instead of one
- *                    bulk copy per row) when the geometry meets the TMA rules
+ *                    2: as 1, and tiles whose two sides differ in order (one
+ *                    token-major, one head-major) are moved with tiled TMA loads
+ *                    or stores through a tensor map of the token-major side (one
+ *                    per head instead of one bulk copy per row) when the
+ *                    geometry meets the TMA rules
  *   "stages"         variant 1: shared-memory stages per CTA, 2..16 (default 3);
  *                    stages x "tile_bytes" must fit in 220 KiB
  *   "dry_run"        1: pdkv_plan_create builds host-only plans (no CUDA call is

@@ -23,6 +23,10 @@
 // The innermost coordinate of every load is 0 (16-byte rule), stage pieces are
 // 128-byte aligned, and a box may over-read past a ragged tile (reads only;
 // out-of-range rows are zero-filled by the hardware and never stored).
+// The opposite direction (head-major source, token-major destination) uses the
+// same map for tiled *stores*: the stage is filled by one contiguous run per
+// head and one tiled store per head scatters its T rows; a ragged tile (fewer
+// than T tokens) must not write a full box and falls back to per-row stores.
 //
 // Every wait is bounded: after kSpinLimit failed polls the warp records an
 // error word, drains its own stores and returns.
@@ -81,6 +85,14 @@ __device__ __forceinline__ void tensor_g2s(void *sdst, const CUtensorMap *map, i
         "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(head), "r"(tok_row), "r"(smem_u32(bar))
         : "memory");
 }
+// Tiled 3-D store of a dense [T][D] piece to the box at (0, head, token row); never negative coordinates.
+__device__ __forceinline__ void tensor_s2g(const CUtensorMap *map, int head, int tok_row, const void *ssrc)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(
+                     reinterpret_cast<uint64_t>(map)),
+                 "r"(0), "r"(head), "r"(tok_row), "r"(smem_u32(ssrc))
+                 : "memory");
+}
 __device__ __forceinline__ void bulk_s2g(void *gdst, const void *ssrc, uint32_t bytes)
 {
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(ssrc)),
@@ -101,10 +113,11 @@ struct Item {
 
 __global__ void __launch_bounds__(32)
 bulk_tiles_kernel(const CopyParams p, const int stages, const uint32_t stage_bytes,
-                  const __grid_constant__ CUtensorMap src_map, const int map_tokens)
+                  const __grid_constant__ CUtensorMap tok_map, const int map_tokens)
 {
-    // map_tokens > 0: src_map describes the source as [token row][head][dim] and its box holds
-    // map_tokens tokens of one head; used for token-major -> head-major tiles only
+    // map_tokens > 0: tok_map describes the token-major side (source or destination) as
+    // [token row][head][dim] and its box holds map_tokens tokens of one head; used for tiles
+    // whose two sides differ in order
     extern __shared__ __align__(128) unsigned char smem[];
     uint64_t *full = reinterpret_cast<uint64_t *>(smem);
     unsigned char *data = smem + kBarrierBytes;
@@ -117,8 +130,9 @@ bulk_tiles_kernel(const CopyParams p, const int stages, const uint32_t stage_byt
     const bool src_flat = p.src.head_stride == p.row_bytes && p.src.tok_stride == hrow;
     const bool dst_flat = p.dst.head_stride == p.row_bytes && p.dst.tok_stride == hrow;
     const uint32_t m_H = div_magic(H);
-    const bool tiled = map_tokens > 0 && src_tok_major && !dst_tok_major;
-    const uint32_t piece = tiled ? (uint32_t)map_tokens * row : 0;   // stage bytes per head
+    const bool tiled = map_tokens > 0 && src_tok_major && !dst_tok_major;       // tiled loads
+    const bool tiled_out = map_tokens > 0 && !src_tok_major && dst_tok_major;   // tiled stores
+    const uint32_t piece = (tiled || tiled_out) ? (uint32_t)map_tokens * row : 0;   // stage bytes per head
 
     if (lane == 0) {
         for (int i = 0; i < stages; ++i) mbar_init(full + i, 1);
@@ -175,12 +189,17 @@ bulk_tiles_kernel(const CopyParams p, const int stages, const uint32_t stage_byt
             if (lane == 0) mbar_arrive_expect(bar, H * piece);
             __syncwarp();
             const int tok_row = (int)(it.s_base / hrow);
-            for (uint32_t hd = lane; hd < H; hd += 32) tensor_g2s(st + (size_t)hd * piece, &src_map, (int)hd, tok_row, bar);
+            for (uint32_t hd = lane; hd < H; hd += 32) tensor_g2s(st + (size_t)hd * piece, &tok_map, (int)hd, tok_row, bar);
             return;
         }
         if (lane == 0) mbar_arrive_expect(bar, bytes);
         __syncwarp();
         const char *src = p.src.base + it.s_base;
+        if (tiled_out) {                    // stage [head][map_tokens][row]: one contiguous run per head
+            const uint32_t run = it.ntok * row;
+            for (uint32_t hd = lane; hd < H; hd += 32) bulk_g2s(st + (size_t)hd * piece, src + hd * p.src.head_stride, run, bar);
+            return;
+        }
         if (src_flat && dst_flat) {                     // one contiguous run on both sides
             if (lane == 0) bulk_g2s(st, src, bytes, bar);
         } else if (src_tok_major == dst_tok_major) {    // same order: one run per head (or per token)
@@ -230,7 +249,18 @@ bulk_tiles_kernel(const CopyParams p, const int stages, const uint32_t stage_byt
             }
             return;
         }
-        if (dst_flat) {
+        if (tiled_out) {
+            if (it.ntok == (uint32_t)map_tokens) {      // a full box per head
+                const int tok_row = (int)(it.d_base / hrow);
+                for (uint32_t hd = lane; hd < H; hd += 32) tensor_s2g(&tok_map, (int)hd, tok_row, st + (size_t)hd * piece);
+            } else {                                    // ragged tile: row by row, nothing past its end
+                const uint32_t rows = it.ntok * H;
+                for (uint32_t r = lane; r < rows; r += 32) {
+                    const uint32_t tk = fast_div(r, m_H), hd = r - tk * H;
+                    bulk_s2g(dst + tk * p.dst.tok_stride + hd * p.dst.head_stride, st + (size_t)hd * piece + (size_t)tk * row, row);
+                }
+            }
+        } else if (dst_flat) {
             if (lane == 0) bulk_s2g(dst, st, it.ntok * H * row);
         } else if (dst_tok_major) {         // token-major with gaps between tokens cannot occur for our sides,
             for (uint32_t tk = lane; tk < it.ntok; tk += 32)   // but keep it correct: one run per token
@@ -297,17 +327,18 @@ EncodeTiled encode_tiled()
     return fn;
 }
 
-// Tensor map of a token-major side viewed as [token rows][H][D]; box = (D, 1, tokens).
+// Tensor map of a token-major side (a block-major pool or the contiguous buffer, flat
+// [token rows][H][D]); box = (D, 1, tokens).
 // Returns false when the geometry does not meet the TMA rules (the caller then
 // uses per-row bulk copies).
-bool make_source_map(const CopyParams &p, int elem_bytes, int tokens, CUtensorMap *out)
+bool make_token_major_map(const CopyParams &p, const Side &side, int elem_bytes, int tokens, CUtensorMap *out)
 {
     const int64_t row = p.row_bytes, hrow = (int64_t)p.H * row;
     if (elem_bytes != 1 && elem_bytes != 2 && elem_bytes != 4 && elem_bytes != 8) return false;
     const int64_t D = row / elem_bytes;
-    const int64_t rows = p.src.size / hrow;
+    const int64_t rows = side.size / hrow;
     if (!encode_tiled() || D < 1 || D > 256 || tokens < 1 || tokens > 256 || row % 16 || rows < 1 ||
-        rows > 0x7FFFFFFFll || ((int64_t)tokens * row) % 128 || (reinterpret_cast<uintptr_t>(p.src.base) & 15u) ||
+        rows > 0x7FFFFFFFll || ((int64_t)tokens * row) % 128 || (reinterpret_cast<uintptr_t>(side.base) & 15u) ||
         hrow >= (1ll << 40))
         return false;
     const CUtensorMapDataType dt = elem_bytes == 1   ? CU_TENSOR_MAP_DATA_TYPE_UINT8
@@ -318,7 +349,7 @@ bool make_source_map(const CopyParams &p, int elem_bytes, int tokens, CUtensorMa
     const cuuint64_t strides[2] = {(cuuint64_t)row, (cuuint64_t)hrow};   // bytes, dimensions 1 and 2
     const cuuint32_t box[3] = {(cuuint32_t)D, 1u, (cuuint32_t)tokens};
     const cuuint32_t estr[3] = {1u, 1u, 1u};
-    return encode_tiled()(out, dt, 3, p.src.base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return encode_tiled()(out, dt, 3, side.base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                           CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -335,9 +366,12 @@ cudaError_t launch_bulk(const CopyParams &p, const LaunchConfig &cfg, cudaStream
     int map_tokens = 0;
     const bool src_tok_major = p.src.tok_stride >= p.src.head_stride;
     const bool dst_tok_major = p.dst.tok_stride >= p.dst.head_stride;
-    if (cfg.variant == 2 && src_tok_major && !dst_tok_major) {
-        const int tokens = (int)(cfg.max_tile_bytes / ((int64_t)p.H * p.row_bytes));
-        if (make_source_map(p, cfg.elem_bytes, tokens, &map)) map_tokens = tokens;
+    if (cfg.variant == 2 && src_tok_major != dst_tok_major) {
+        const Side &side = src_tok_major ? p.src : p.dst;
+        const int64_t hrow = (int64_t)p.H * p.row_bytes;
+        const bool side_flat = side.head_stride == p.row_bytes && side.tok_stride == hrow;
+        const int tokens = (int)(cfg.max_tile_bytes / hrow);
+        if (side_flat && make_token_major_map(p, side, cfg.elem_bytes, tokens, &map)) map_tokens = tokens;
     }
     const int stages = cfg.stages;
     const size_t smem = kBarrierBytes + (size_t)stages * stage_bytes;
