@@ -265,6 +265,7 @@ def step_bytes_of(w):
 def cpu_baseline(w, src_t, budget_s=20.0):
     """Time the CPU checker, as it stands, on the first requests of the batch."""
     import numpy as np
+    import torch
 
     from oracle import pdkv_oracle as O
     from paper_2408_08147_b200 import workloads as W
@@ -278,7 +279,7 @@ def cpu_baseline(w, src_t, budget_s=20.0):
     while n > 1 and 6 * int(w.batch.seq_len[:n].sum()) * tok_bytes / 0.4e9 > 2 * budget_s:
         n -= 1
     sub, s_ids, _ = W.compact_subproblem(w, range(n))
-    src_np = W.gather_blocks(src_t.view(__import__("torch").int16), w.src, s_ids).cpu().numpy().view(np.uint16)
+    src_np = W.gather_blocks(src_t.view(torch.int16), w.src, s_ids).cpu().numpy().view(np.uint16)
     dst_np = W.sentinel_pool_numpy(sub.dst)
     buf_np = np.zeros(O.buffer_elems(sub.batch, sub.dst.block_tokens, sub.src), np.uint16)
     threads = min(cores, n)
@@ -288,7 +289,7 @@ def cpu_baseline(w, src_t, budget_s=20.0):
     nbytes = step_bytes_of(sub)
     # the same checker on one request with one thread, for a per-core figure
     one, one_ids, _ = W.compact_subproblem(w, [0])
-    one_src = W.gather_blocks(src_t.view(__import__("torch").int16), w.src, one_ids).cpu().numpy().view(np.uint16)
+    one_src = W.gather_blocks(src_t.view(torch.int16), w.src, one_ids).cpu().numpy().view(np.uint16)
     one_dst = W.sentinel_pool_numpy(one.dst)
     one_buf = np.zeros(O.buffer_elems(one.batch, one.dst.block_tokens, one.src), np.uint16)
     t1 = time.perf_counter()
