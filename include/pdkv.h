@@ -140,6 +140,21 @@ int pdkv_pool_destroy(pdkv_pool *pool);
 int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst,
                      int32_t skip_granule_tokens, const pdkv_batch_desc *batch,
                      void *stream, pdkv_plan **out);
+/* As pdkv_plan_create(), but the plan's device arrays (a 256-byte status area
+ * and the tile lists) are placed in `workspace` (device, 16-byte aligned,
+ * workspace_bytes long) instead of a cudaMalloc'ed block: creation then
+ * allocates nothing on the device and pdkv_plan_destroy() frees nothing, which
+ * takes cudaMalloc/cudaFree (about 0.3 ms each) off the path of engines that
+ * build a plan per transfer.  The workspace belongs to the caller and must stay
+ * untouched until the plan is destroyed.  `needed_bytes` (optional) receives
+ * the size the batch needs; if the workspace is smaller the call returns
+ * PDKV_ERR_BUFFER_TOO_SMALL and creates nothing.  workspace == NULL behaves
+ * exactly like pdkv_plan_create(). */
+int pdkv_plan_create_in(const pdkv_pool *src, const pdkv_pool *dst,
+                        int32_t skip_granule_tokens, const pdkv_batch_desc *batch,
+                        void *workspace, size_t workspace_bytes, size_t *needed_bytes,
+                        void *stream, pdkv_plan **out);
+
 /* Frees the plan and its device arrays.  Call it once the work enqueued with
  * the plan has completed (its kernels read the tile lists). */
 int pdkv_plan_destroy(pdkv_plan *plan);

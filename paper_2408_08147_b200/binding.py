@@ -37,7 +37,7 @@ PDKV_OP_TRANSFER = 2
 PDKV_OP_BLOCKWISE = 3  # only for pdkv_plan_launches
 
 EXPORTS = (
-    "pdkv_pool_bytes", "pdkv_pool_create", "pdkv_pool_destroy", "pdkv_plan_create",
+    "pdkv_pool_bytes", "pdkv_pool_create", "pdkv_pool_destroy", "pdkv_plan_create", "pdkv_plan_create_in",
     "pdkv_plan_destroy", "pdkv_plan_buffer", "pdkv_plan_traffic", "pdkv_pack", "pdkv_unpack",
     "pdkv_transfer", "pdkv_transfer_noalloc", "pdkv_transfer_blockwise", "pdkv_plan_launches", "pdkv_plan_tiles",
     "pdkv_plan_status", "pdkv_upload_blocks", "pdkv_download_blocks", "pdkv_plan_block_bytes",
@@ -91,6 +91,8 @@ def lib() -> C.CDLL:
     L.pdkv_pool_create.argtypes = [C.POINTER(pdkv_pool_desc), vp, C.c_size_t, C.c_int, C.POINTER(vp)]
     L.pdkv_pool_destroy.argtypes = [vp]
     L.pdkv_plan_create.argtypes = [vp, vp, i32, C.POINTER(pdkv_batch_desc), vp, C.POINTER(vp)]
+    L.pdkv_plan_create_in.argtypes = [vp, vp, i32, C.POINTER(pdkv_batch_desc), vp, C.c_size_t,
+                                      C.POINTER(C.c_size_t), vp, C.POINTER(vp)]
     L.pdkv_plan_destroy.argtypes = [vp]
     L.pdkv_plan_buffer.argtypes = [vp, C.POINTER(C.c_size_t), C.POINTER(C.POINTER(i64))]
     L.pdkv_plan_traffic.argtypes = [vp, C.c_int, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
@@ -181,6 +183,24 @@ def pdkv_plan_create(src_pool: Optional[int], dst_pool: Optional[int], skip_gran
                                   skip_granule_tokens, C.byref(b.desc), C.c_void_p(stream),
                                   C.byref(out)), "pdkv_plan_create")
     return out.value
+
+
+def pdkv_plan_create_in(src_pool: Optional[int], dst_pool: Optional[int], skip_granule_tokens: int,
+                        seq_len, src_tbl_off=None, src_tbl=None, dst_tbl_off=None, dst_tbl=None,
+                        dst_skip=None, workspace_ptr: int = 0, workspace_bytes: int = 0, stream: int = 0):
+    """Plan whose device arrays live in caller-provided device memory.
+    Returns (plan, needed_bytes); raises PdkvError(BUFFER_TOO_SMALL) with
+    ``.needed_bytes`` set when the workspace is too small."""
+    b = _BatchArrays(seq_len, src_tbl_off, src_tbl, dst_tbl_off, dst_tbl, dst_skip)
+    out, need = C.c_void_p(), C.c_size_t()
+    rc = lib().pdkv_plan_create_in(C.c_void_p(src_pool), C.c_void_p(dst_pool), skip_granule_tokens,
+                                   C.byref(b.desc), C.c_void_p(workspace_ptr), workspace_bytes, C.byref(need),
+                                   C.c_void_p(stream), C.byref(out))
+    if rc != PDKV_OK:
+        err = PdkvError(rc, "pdkv_plan_create_in")
+        err.needed_bytes = int(need.value)
+        raise err
+    return out.value, int(need.value)
 
 
 def pdkv_plan_destroy(plan: int) -> None:

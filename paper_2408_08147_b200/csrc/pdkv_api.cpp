@@ -75,6 +75,7 @@ struct pdkv_plan {
     // maximal runs of consecutive block ids: prefill blocks the batch reads, decode blocks it writes
     std::vector<std::pair<int64_t, int64_t>> src_runs, dst_runs;  // (first id, count)
     void *dev_mem = nullptr;
+    bool owns_dev_mem = true;   // false: dev_mem is a caller-provided workspace
     unsigned long long *dev_status = nullptr;
     int vec_bytes = 16;
     int64_t max_tile_bytes = 0;
@@ -367,7 +368,15 @@ int pdkv_pool_destroy(pdkv_pool *pool)
 int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip_granule_tokens,
                      const pdkv_batch_desc *batch, void *stream, pdkv_plan **out)
 {
+    return pdkv_plan_create_in(src, dst, skip_granule_tokens, batch, nullptr, 0, nullptr, stream, out);
+}
+
+int pdkv_plan_create_in(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip_granule_tokens,
+                        const pdkv_batch_desc *batch, void *workspace, size_t workspace_bytes,
+                        size_t *needed_bytes, void *stream, pdkv_plan **out)
+{
     if (out) *out = nullptr;
+    if (needed_bytes) *needed_bytes = 0;
     if (!out || !batch || (!src && !dst)) return PDKV_ERR_INVALID_ARG;
     if (batch->n_req < 0 || (batch->n_req > 0 && !batch->seq_len)) return PDKV_ERR_INVALID_ARG;
     if (src && dst) {
@@ -526,6 +535,12 @@ int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip_gr
             pl->mean_tile_bytes[op] = pl->tiles[op].empty() ? 0 : sum / (int64_t)pl->tiles[op].size();
         }
 
+        // device bytes of the plan: [status words][pack tiles][unpack tiles][transfer tiles]
+        const size_t head = 256;
+        size_t total = head;
+        for (int op = 0; op < 3; ++op) total += pl->tiles[op].size() * sizeof(Tile);
+        if (needed_bytes) *needed_bytes = total;
+
         if (pdkv::tunables().dry_run || g_host_only_plan) {  // host-only plan: tile lists can be inspected, nothing can launch
             hold.p = nullptr;
             *out = pl;
@@ -538,11 +553,15 @@ int pdkv_plan_create(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip_gr
         // (cudaGetDeviceProperties costs milliseconds; one attribute query does not)
         cudaError_t e = cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, pl->device);
         if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
-        const size_t head = 256;
-        size_t total = head;
-        for (int op = 0; op < 3; ++op) total += pl->tiles[op].size() * sizeof(Tile);
-        e = cudaMalloc(&pl->dev_mem, total);
-        if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc");
+        if (workspace) {  // caller-provided device memory: nothing is allocated or freed
+            if (!aligned16(workspace)) return PDKV_ERR_INVALID_ARG;
+            if (workspace_bytes < total) return PDKV_ERR_BUFFER_TOO_SMALL;
+            pl->dev_mem = workspace;
+            pl->owns_dev_mem = false;
+        } else {
+            e = cudaMalloc(&pl->dev_mem, total);
+            if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc");
+        }
         cudaStream_t st = static_cast<cudaStream_t>(stream);
         e = cudaMemsetAsync(pl->dev_mem, 0, head, st);
         if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
@@ -572,7 +591,7 @@ int pdkv_plan_destroy(pdkv_plan *plan)
 {
     if (!plan) return PDKV_OK;
     int rc = PDKV_OK;
-    if (plan->dev_mem) {
+    if (plan->dev_mem && plan->owns_dev_mem) {
         DeviceGuard guard(plan->device);
         cudaError_t e = cudaFree(plan->dev_mem);
         if (e != cudaSuccess) rc = cuda_fail(e, "cudaFree");

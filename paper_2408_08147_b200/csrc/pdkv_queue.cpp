@@ -16,6 +16,7 @@ struct Slot {
     cudaStream_t stream = nullptr;
     cudaEvent_t done = nullptr;
     pdkv_plan *plan = nullptr;
+    void *workspace = nullptr;   // device memory for the slot's plan, reused across tickets
     int64_t ticket = -1;   // -1: free
 };
 
@@ -32,6 +33,8 @@ struct pdkv_queue {
 };
 
 namespace {
+
+constexpr size_t kSlotWorkspaceBytes = 1 << 20;   // tile lists of ~14k tiles; larger batches fall back to cudaMalloc
 
 Slot *find(pdkv_queue *q, int64_t ticket)
 {
@@ -64,6 +67,7 @@ int pdkv_queue_create(const pdkv_pool *src, const pdkv_pool *dst, int device, in
         for (Slot &s : q->slots) {
             if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking);
             if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaMalloc(&s.workspace, kSlotWorkspaceBytes);
         }
         if (e != cudaSuccess) {
             const int rc = pdkv::report_cuda_error(e, "queue set-up");
@@ -98,7 +102,10 @@ int pdkv_queue_submit(pdkv_queue *q, const pdkv_batch_desc *batch, const void *h
     } else {
         DevGuard guard(q->device);
         if (guard.err != cudaSuccess) return pdkv::report_cuda_error(guard.err, "cudaSetDevice");
-        rc = pdkv_plan_create(q->src, q->dst, 0, batch, slot->stream, &slot->plan);
+        rc = pdkv_plan_create_in(q->src, q->dst, 0, batch, slot->workspace, kSlotWorkspaceBytes, nullptr,
+                                 slot->stream, &slot->plan);
+        if (rc == PDKV_ERR_BUFFER_TOO_SMALL)   // a batch with more tiles than the slot's workspace holds
+            rc = pdkv_plan_create(q->src, q->dst, 0, batch, slot->stream, &slot->plan);
         if (rc != PDKV_OK) return rc;
         if (host_src_pool) rc = pdkv_upload_blocks(slot->plan, host_src_pool, slot->stream);
         if (rc == PDKV_OK) rc = pdkv_transfer(slot->plan, 0, pdkv::plan_num_layers(slot->plan), slot->stream);
@@ -192,6 +199,7 @@ int pdkv_queue_destroy(pdkv_queue *q)
             if (s.stream) cudaStreamSynchronize(s.stream);
             if (s.plan) pdkv_plan_destroy(s.plan);
             if (s.done) cudaEventDestroy(s.done);
+            if (s.workspace) cudaFree(s.workspace);
             if (s.stream && cudaStreamDestroy(s.stream) != cudaSuccess) rc = PDKV_ERR_CUDA;
         }
     }

@@ -405,3 +405,33 @@ def test_sender_only_and_receiver_only_plans(oracle, idx, kw):
     finally:
         sender.close()
         receiver.close()
+
+
+def test_plan_in_caller_workspace(oracle):
+    """pdkv_plan_create_in keeps the plan's device arrays in memory the caller
+    owns: too small a workspace is refused with the needed size, a sufficient one
+    gives the same bytes as an allocating plan, and the workspace can be reused."""
+    w = W.make_config(3, num_layers=2, n_req=8, max_len=900)
+    b = w.batch
+    src = W.fill_pool_numpy(w.src, w.seed)
+    sent = W.sentinel_pool_numpy(w.dst)
+    want = sent.copy()
+    oracle.transfer(w.src, src, w.dst, want, b)
+    src_t, dst_t = dev(src), dev(sent)
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    ps = B.pdkv_pool_create(B.desc_of(w.src), src_t.data_ptr(), src_t.numel(), 0)
+    pd = B.pdkv_pool_create(B.desc_of(w.dst), dst_t.data_ptr(), dst_t.numel(), 0)
+    args = (ps, pd, 0, b.seq_len, b.src_tbl_off, b.src_tbl, b.dst_tbl_off, b.dst_tbl, b.dst_skip)
+    with pytest.raises(B.PdkvError) as e:
+        B.pdkv_plan_create_in(*args, workspace_ptr=ws.data_ptr(), workspace_bytes=512)
+    assert e.value.status == B.PDKV_ERR_BUFFER_TOO_SMALL and e.value.needed_bytes > 512
+    for _ in range(2):                                   # the same workspace, two plans in a row
+        plan, need = B.pdkv_plan_create_in(*args, workspace_ptr=ws.data_ptr(), workspace_bytes=ws.numel())
+        assert need == e.value.needed_bytes
+        B.pdkv_transfer(plan, 0, w.src.num_layers)
+        B.pdkv_plan_status(plan)
+        assert np.array_equal(host(dst_t), want)
+        B.pdkv_plan_destroy(plan)
+        dst_t.copy_(dev(sent)); torch.cuda.synchronize()
+    B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)

@@ -306,3 +306,15 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
         B.lib()
     with pytest.raises(ImportError):
         B.pdkv_pool_bytes(B.make_desc(0, 1, 1, 8, 2, 4, 2))
+
+
+def test_workspace_plans_report_their_size():
+    w = W.make_config(3, num_layers=2, n_req=6, max_len=700)
+    ps, pd = _pools(w)
+    b = w.batch
+    plan, need = B.pdkv_plan_create_in(ps, pd, 0, b.seq_len, b.src_tbl_off, b.src_tbl, b.dst_tbl_off, b.dst_tbl,
+                                       b.dst_skip)
+    tiles = sum(len(B.pdkv_plan_tiles(plan, op)) for op in range(3))
+    assert need == 256 + 24 * tiles
+    B.pdkv_plan_destroy(plan)
+    B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
