@@ -542,12 +542,15 @@ def e2e_leg(args, w, src_t, dst_t, buf_t, stream, step_bytes, torch, B, Transfer
     groups = [W.slice_batch(w.batch, cuts[i], cuts[i + 1]) for i in range(n_groups)]
     streams = [torch.cuda.Stream() for _ in range(min(3, n_groups))]
     setup = torch.cuda.Stream()
+    # one preallocated workspace per group for its plan: no cudaMalloc / cudaFree inside a step
+    spaces = [torch.empty(4 << 20, dtype=torch.uint8, device=dev) for _ in range(n_groups)]
 
     def one():
         sessions, at, up, down = [], 0, 0, 0
         for g, part in enumerate(groups):
             st = streams[g % len(streams)].cuda_stream
-            s = TransferSession(w.src, src_t, w.dst, dst_t, part, setup.cuda_stream)   # plan: tables from host
+            s = TransferSession(w.src, src_t, w.dst, dst_t, part, setup.cuda_stream,   # plan: tables from host
+                                workspace_t=spaces[g])
             piece = buf_t[at:at + s.buffer_bytes] if s.buffer_bytes else buf_t[:16]
             at += s.buffer_bytes
             s.upload_blocks(h_src, st)      # pdkv_upload_blocks: H2D of the group's prefill blocks
@@ -577,7 +580,7 @@ def e2e_leg(args, w, src_t, dst_t, buf_t, stream, step_bytes, torch, B, Transfer
     del h_src, h_dst
     return {"value": units / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms, "steps": steps,
             "h2d_bytes_per_step": int(up_down[0]), "d2h_bytes_per_step": int(up_down[1]),
-            "includes": "pdkv_plan_create (tables from host arrays), pdkv_upload_blocks from a pinned host image of "
+            "includes": "pdkv_plan_create_in (tables from host arrays, preallocated workspaces), pdkv_upload_blocks from a pinned host image of "
                         "the prefill pool, pack, unpack, fused, pdkv_download_blocks into a pinned host image of "
                         "the decode pool; wall clock",
             "pipeline": f"{n_groups} request groups over {len(streams)} streams"}

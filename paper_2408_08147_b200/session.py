@@ -20,7 +20,10 @@ class TransferSession:
     """
 
     def __init__(self, src_geom, src_t, dst_geom, dst_t, batch, stream: int = 0,
-                 skip_granule_tokens: int = 0):
+                 skip_granule_tokens: int = 0, workspace_t=None):
+        """``workspace_t``: optional flat torch CUDA tensor that receives the plan's
+        device arrays (no cudaMalloc / cudaFree for this session); it must outlive
+        the session and not be shared with another live session."""
         self.src_geom, self.dst_geom, self.batch = src_geom, dst_geom, batch
         self.src_t, self.dst_t = src_t, dst_t
         self.stream = stream
@@ -34,13 +37,20 @@ class TransferSession:
                 self.dst_pool = B.pdkv_pool_create(B.desc_of(dst_geom), dst_t.data_ptr(),
                                                    dst_t.numel() * dst_t.element_size(),
                                                    dst_t.device.index or 0)
-            self.plan = B.pdkv_plan_create(
-                self.src_pool, self.dst_pool, skip_granule_tokens, batch.seq_len,
-                batch.src_tbl_off if src_t is not None else None,
-                batch.src_tbl if src_t is not None else None,
-                batch.dst_tbl_off if (dst_t is not None or batch.dst_skip is not None) else None,
-                batch.dst_tbl if dst_t is not None else None,
-                batch.dst_skip, stream)
+            tables = (batch.seq_len,
+                      batch.src_tbl_off if src_t is not None else None,
+                      batch.src_tbl if src_t is not None else None,
+                      batch.dst_tbl_off if (dst_t is not None or batch.dst_skip is not None) else None,
+                      batch.dst_tbl if dst_t is not None else None,
+                      batch.dst_skip)
+            if workspace_t is None:
+                self.plan = B.pdkv_plan_create(self.src_pool, self.dst_pool, skip_granule_tokens, *tables,
+                                               stream=stream)
+            else:
+                self.plan, _ = B.pdkv_plan_create_in(
+                    self.src_pool, self.dst_pool, skip_granule_tokens, *tables,
+                    workspace_ptr=workspace_t.data_ptr(),
+                    workspace_bytes=workspace_t.numel() * workspace_t.element_size(), stream=stream)
         except Exception:
             self.close()
             raise
