@@ -318,3 +318,39 @@ def test_workspace_plans_report_their_size():
     assert need == 256 + 24 * tiles
     B.pdkv_plan_destroy(plan)
     B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
+
+
+def test_tile_offsets_in_petabyte_pools_need_64_bits():
+    """Offsets are 64-bit end to end: pools far beyond any GPU (dry-run plans only)
+    give tile offsets equal to exact Python integer arithmetic."""
+    L, H, D, E, Bp, Bd = 80, 8, 128, 2, 64, 128
+    nb_src, nb_dst = 50_000_000, 30_000_000
+    gs = W.Geometry(W.BLOCK_MAJOR, L, H, D, E, Bp, nb_src)
+    gd = W.Geometry(W.LAYER_MAJOR, L, H, D, E, Bd, nb_dst)
+    assert gs.num_bytes() > 2 ** 49
+    lens = np.array([200, 64, 129], np.int32)
+    n_s = -(-lens.astype(np.int64) // Bp); n_d = -(-lens.astype(np.int64) // Bd)
+    rng = np.random.default_rng(5)
+    src_tbl = rng.choice(np.arange(nb_src - 1000, nb_src), size=int(n_s.sum()), replace=False).astype(np.int32)
+    dst_tbl = rng.choice(np.arange(nb_dst - 1000, nb_dst), size=int(n_d.sum()), replace=False).astype(np.int32)
+    off_s = np.concatenate([[0], np.cumsum(n_s)]).astype(np.int64)
+    off_d = np.concatenate([[0], np.cumsum(n_d)]).astype(np.int64)
+    ps = B.pdkv_pool_create(B.desc_of(gs), FAKE_BASE, gs.num_bytes(), 0)
+    pd = B.pdkv_pool_create(B.desc_of(gd), 0x100000000000000, gd.num_bytes(), 0)
+    B.pdkv_tune("tile_bytes", 32768)
+    plan = B.pdkv_plan_create(ps, pd, 0, lens, off_s, src_tbl, off_d, dst_tbl)
+    row, hrow = D * E, H * D * E
+    tiles = B.pdkv_plan_tiles(plan, B.PDKV_OP_TRANSFER)
+    copy = tiles[tiles["src_off"] >= 0]
+    want = []
+    for r in range(3):
+        t = 0
+        while t < lens[r]:
+            end = min(int(lens[r]), (t // Bp + 1) * Bp, (t // Bd + 1) * Bd, t + 32768 // hrow)
+            bs, bd = int(src_tbl[off_s[r] + t // Bp]), int(dst_tbl[off_d[r] + t // Bd])
+            want.append((bs * (2 * L * Bp * hrow) + (t % Bp) * hrow, bd * (H * Bd * row) + (t % Bd) * row, end - t))
+            t = end
+    got = [(int(a), int(b), int(c)) for a, b, c in zip(copy["src_off"], copy["dst_off"], copy["ntok"])]
+    assert got == want and max(a for a, _, _ in got) > 2 ** 49
+    B.pdkv_plan_destroy(plan)
+    B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
