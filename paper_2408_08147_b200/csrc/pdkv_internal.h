@@ -1,6 +1,7 @@
 // Internal declarations shared by the host planner and the kernel launchers.
 #pragma once
 
+#include <atomic>
 #include <cstdint>
 #include <vector>
 
@@ -86,21 +87,22 @@ struct DeviceGuard {
     DeviceGuard &operator=(const DeviceGuard &) = delete;
 };
 
+// Process-wide settings; atomics because pdkv_tune may race with launches on other threads.
 struct Tunables {
-    int64_t tile_bytes = 32768;
-    int64_t ctas_per_sm = 2;
-    int64_t max_ctas = 0;
-    int64_t threads = 0;   // 0: chosen with unroll, per class of copy
-    int64_t unroll = 0;    // 0: chosen per class of copy
-    int64_t vec32 = 1;
-    int64_t lc_fastest = 0;
-    int64_t group_threads = 0;   // 0: sized from the plan's mean tile
-    int64_t chunked = 0;
-    int64_t debug_bounds = 0;
-    int64_t debug_shrink = 0;   // with debug_bounds: treat the last N bytes of each side as out of range
-    int64_t variant = 0;
-    int64_t stages = 3;
-    int64_t dry_run = 0;
+    std::atomic<int64_t> tile_bytes{32768};
+    std::atomic<int64_t> ctas_per_sm{2};
+    std::atomic<int64_t> max_ctas{0};
+    std::atomic<int64_t> threads{0};   // 0: chosen with unroll, per class of copy
+    std::atomic<int64_t> unroll{0};    // 0: chosen per class of copy
+    std::atomic<int64_t> vec32{1};
+    std::atomic<int64_t> lc_fastest{0};
+    std::atomic<int64_t> group_threads{0};   // 0: sized from the plan's mean tile
+    std::atomic<int64_t> chunked{0};
+    std::atomic<int64_t> debug_bounds{0};
+    std::atomic<int64_t> debug_shrink{0};   // with debug_bounds: treat the last N bytes of each side as out of range
+    std::atomic<int64_t> variant{0};
+    std::atomic<int64_t> stages{3};
+    std::atomic<int64_t> dry_run{0};
 };
 Tunables &tunables();
 
