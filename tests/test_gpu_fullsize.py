@@ -3,9 +3,10 @@ benchmark times (library defaults).  Pools of 8-50 GiB cannot be replayed on the
 CPU checker in one piece, so requests are checked as self-contained sub-problems
 (their blocks gathered out of both pools): the checker computes buffer and
 decode blocks for the sub-problem and the GPU's bytes for those requests must be
-identical.  Configs 2 and 3 are checked in full this way (every request, hence
-every owned byte); configs 4 and 5 on a seeded sample of requests.  Bytes nobody may touch
-(resident decode blocks, the buffer's slack) are compared with the sentinel."""
+identical.  Configs 2 to 5 are checked in full this way (every request, hence
+every owned byte; config 5 at both ends of its prefill-block sweep).  Bytes nobody
+may touch (resident decode blocks, the buffer's slack, the prefill pool itself) are
+compared with the sentinel or a checksum."""
 import numpy as np
 import pytest
 
@@ -39,20 +40,80 @@ def _np16(t):
     return t.cpu().numpy().view(np.uint16)
 
 
+def _checksum(t):
+    """Order-independent 64-bit sum of a pool's 32-bit words (cheap "was it written?" test)."""
+    v, total, step = t.view(torch.int32), 0, 1 << 28
+    for i in range(0, v.numel(), step):
+        total += int(v[i:i + step].sum(dtype=torch.int64).item())
+    return total
+
+
+class _Staging:
+    """Pinned host buffers reused for every request group (pageable copies of
+    tens of GiB would dominate the test's run time)."""
+
+    def __init__(self):
+        self.bufs = {}
+
+    def get(self, name, n_bytes):
+        t = self.bufs.get(name)
+        if t is None or t.numel() < n_bytes:
+            self.bufs[name] = t = torch.empty(max(n_bytes, 16), dtype=torch.uint8, pin_memory=True)
+        return t[:n_bytes]
+
+    def to_host(self, name, dev_t):
+        h = self.get(name, dev_t.numel() * dev_t.element_size())
+        h.copy_(dev_t.reshape(-1).view(torch.uint8))
+        torch.cuda.synchronize()
+        return h.numpy().view(np.uint16)
+
+    def host_array(self, name, n_elems):
+        return self.get(name, 2 * n_elems).numpy().view(np.uint16)
+
+    def to_device(self, name, n_elems):
+        return self.get(name, 2 * n_elems).cuda().view(torch.int16)
+
+
+def _checker_in_parallel(call, n_req, n_layers):
+    """Run a checker function over (request, layer range) pieces on all host
+    cores; pieces write disjoint bytes and the C code runs without the GIL."""
+    import os
+    from concurrent.futures import ThreadPoolExecutor
+
+    workers = os.cpu_count() or 1
+    cuts = max(1, min(n_layers, -(-2 * workers // max(1, n_req))))
+    edges = np.linspace(0, n_layers, cuts + 1).astype(int)
+    tasks = [(r, int(edges[i]), int(edges[i + 1])) for r in range(n_req) for i in range(cuts)]
+    with ThreadPoolExecutor(max_workers=workers) as ex:
+        list(ex.map(lambda t: call(layers=(t[1], t[2]), requests=(t[0], t[0] + 1)), tasks))
+
+
 def run_fullsize(oracle, w, n_sample, seed, group=1):
     """n_sample = 0 checks every request (in groups of `group` consecutive
-    requests, one checker thread each); otherwise a seeded sample."""
+    requests); otherwise a seeded sample.
+
+    The four calls (pack + unpack, fused, block-by-block) each get a decode pool
+    of their own while device memory lasts; the request groups are then streamed:
+    gather the group's prefill blocks, run the checker on that sub-problem on the
+    host, send its buffer and decode blocks back and compare on the device with
+    torch.equal.  Host memory stays bounded by one group whatever the batch size.
+    With fewer than three decode pools the remaining calls run in a further pass."""
     from paper_2408_08147_b200.session import TransferSession
 
     import gc
 
     gc.collect()
     torch.cuda.empty_cache()        # earlier tests' pools sit in torch's cache, not in the driver's free list
-    need = w.src.num_bytes() + 2 * w.dst.num_bytes()
-    free, _ = torch.cuda.mem_get_info()
-    if need * 1.1 > free:
-        pytest.skip(f"needs {need >> 30} GiB of device memory")
     b = w.batch
+    G = w.dst.block_tokens
+    L = w.src.num_layers
+    payload = int(oracle.buffer_elems(b, G, w.src)) * w.src.elem_bytes
+    free, _ = torch.cuda.mem_get_info()
+    headroom = 12 << 30             # gathered sub-pools and torch's workspace
+    fixed = w.src.num_bytes() + payload + SLACK
+    n_pools = int(min(3, (free - headroom - fixed) // w.dst.num_bytes()))
+    if n_pools < 1:
+        pytest.skip(f"needs {(fixed + w.dst.num_bytes() + headroom) >> 30} GiB of device memory")
     rng = np.random.default_rng(seed)
     if n_sample == 0:
         groups = [list(range(i, min(i + group, b.n_req))) for i in range(0, b.n_req, group)]
@@ -61,66 +122,70 @@ def run_fullsize(oracle, w, n_sample, seed, group=1):
 
     src_t = torch.empty(w.src.num_bytes(), dtype=torch.uint8, device="cuda")
     W.fill_pool_torch(src_t, w.seed)
-    dst_t = torch.empty(w.dst.num_bytes(), dtype=torch.uint8, device="cuda")
-    _sentinel_fill(dst_t)
+    src_sum = _checksum(src_t)
+    pools = [torch.empty(w.dst.num_bytes(), dtype=torch.uint8, device="cuda") for _ in range(n_pools)]
     stream = torch.cuda.Stream()
     torch.cuda.synchronize()
-    G = w.dst.block_tokens
+    stage = _Staging()
 
-    with TransferSession(w.src, src_t, w.dst, dst_t, b, stream.cuda_stream) as s:
-        assert s.buffer_bytes == sum(s.traffic(B.PDKV_OP_PACK)) // 2
-        buf_t = torch.empty(s.buffer_bytes + SLACK, dtype=torch.uint8, device="cuda")
+    sessions = [TransferSession(w.src, src_t, w.dst, p, b, stream.cuda_stream) for p in pools]
+    try:
+        s0 = sessions[0]
+        assert s0.buffer_bytes == payload == sum(s0.traffic(B.PDKV_OP_PACK)) // 2
+        buf_t = torch.empty(payload + SLACK, dtype=torch.uint8, device="cuda")
         _sentinel_fill(buf_t)
-
-        # expected bytes of every sampled request, from the checker
-        expect = {}
-        for g in groups:
-            sub, s_ids, d_ids = W.compact_subproblem(w, g)
-            sub_src = _np16(W.gather_blocks(src_t.view(torch.int16), w.src, s_ids))
-            want_buf = np.zeros(oracle.buffer_elems(sub.batch, G, sub.src), np.uint16)
-            oracle.pack(sub.src, sub_src, sub.batch, G, want_buf, threads=len(g))
-            want_dst = W.sentinel_pool_numpy(sub.dst)
-            oracle.transfer(sub.src, sub_src, sub.dst, want_dst, sub.batch, threads=len(g))
-            expect[(g[0], g[-1] + 1)] = (want_buf, want_dst, d_ids)
-            assert want_buf.size * 2 == s.request_offsets[g[-1] + 1] - s.request_offsets[g[0]]
-
-        def check_dst(what):
-            for r, (_, want_dst, d_ids) in expect.items():
-                got = _np16(W.gather_blocks(dst_t.view(torch.int16), w.dst, d_ids))
-                assert np.array_equal(got, want_dst), f"{what}: requests {r[0]}..{r[1] - 1}"
-
-        s.pack(buf_t)
-        torch.cuda.synchronize()
-        for (r0, r1), (want_buf, _, _) in expect.items():
-            a, z = int(s.request_offsets[r0]), int(s.request_offsets[r1])
-            assert np.array_equal(_np16(buf_t[a:z]), want_buf), f"pack: requests {r0}..{r1 - 1}"
-        assert bool((buf_t[s.buffer_bytes:].view(torch.int16) == SENT).all()), "pack wrote past the buffer"
-
-        s.unpack(buf_t)
-        torch.cuda.synchronize()
-        check_dst("unpack")
-
-        _sentinel_fill(dst_t)
-        s.transfer()
-        torch.cuda.synchronize()
-        check_dst("fused")
-
-        # resident (skipped) decode blocks keep the sentinel
-        if b.dst_skip is not None:
-            nblk = -(-b.seq_len.astype(np.int64) // G)
-            ids = np.concatenate([b.dst_tbl[b.dst_tbl_off[r]:b.dst_tbl_off[r] + nblk[r]]
-                                  [b.dst_skip[b.dst_tbl_off[r]:b.dst_tbl_off[r] + nblk[r]] != 0]
-                                  for r in range(b.n_req)])
-            assert ids.size > 0
-            for i in range(0, ids.size, 64):
-                blk = W.gather_blocks(dst_t.view(torch.int16), w.dst, ids[i:i + 64])
-                assert bool((blk == SENT).all()), "a resident decode block was written"
-
-        _sentinel_fill(dst_t)
-        s.transfer_blockwise()
-        torch.cuda.synchronize()
-        check_dst("block-by-block baseline")
-    del src_t, dst_t, buf_t, s
+        calls = [("unpack", lambda s: (s.pack(buf_t), s.unpack(buf_t))),
+                 ("fused", lambda s: s.transfer()),
+                 ("block-by-block baseline", lambda s: s.transfer_blockwise())]
+        first_pass = True
+        while calls:
+            now, calls = calls[:n_pools], calls[n_pools:]
+            for (what, call), s, pool in zip(now, sessions, pools):
+                _sentinel_fill(pool)
+                call(s)
+            torch.cuda.synchronize()
+            for g in groups:
+                sub, s_ids, d_ids = W.compact_subproblem(w, g)
+                sub_src = stage.to_host("src", W.gather_blocks(src_t.view(torch.int16), w.src, s_ids))
+                if first_pass:
+                    want_buf = stage.host_array("buf", oracle.buffer_elems(sub.batch, G, sub.src))
+                    want_buf[:] = 0
+                    _checker_in_parallel(lambda **kw: oracle.pack(sub.src, sub_src, sub.batch, G, want_buf, **kw),
+                                         len(g), L)
+                    a, z = int(s0.request_offsets[g[0]]), int(s0.request_offsets[g[-1] + 1])
+                    assert want_buf.size * 2 == z - a
+                    want_dev = stage.to_device("buf", want_buf.size)
+                    assert torch.equal(buf_t[a:z].view(torch.int16), want_dev), f"pack: requests {g[0]}..{g[-1]}"
+                    del want_dev
+                want_dst = stage.host_array("dst", sub.dst.num_elems())
+                want_dst[:] = SENT
+                _checker_in_parallel(lambda **kw: oracle.transfer(sub.src, sub_src, sub.dst, want_dst, sub.batch, **kw),
+                                     len(g), L)
+                want_dev = stage.to_device("dst", want_dst.size)
+                for (what, _), pool in zip(now, pools):
+                    got = W.gather_blocks(pool.view(torch.int16), w.dst, d_ids)
+                    assert torch.equal(got, want_dev), f"{what}: requests {g[0]}..{g[-1]}"
+                    del got
+                del want_dev
+            if first_pass:
+                assert bool((buf_t[payload:].view(torch.int16) == SENT).all()), "pack wrote past the buffer"
+            # resident (skipped) decode blocks keep the sentinel after every call
+            if b.dst_skip is not None:
+                nblk = -(-b.seq_len.astype(np.int64) // G)
+                ids = np.concatenate([b.dst_tbl[b.dst_tbl_off[r]:b.dst_tbl_off[r] + nblk[r]]
+                                      [b.dst_skip[b.dst_tbl_off[r]:b.dst_tbl_off[r] + nblk[r]] != 0]
+                                      for r in range(b.n_req)])
+                assert ids.size > 0
+                for (what, _), pool in zip(now, pools):
+                    for i in range(0, ids.size, 64):
+                        blk = W.gather_blocks(pool.view(torch.int16), w.dst, ids[i:i + 64])
+                        assert bool((blk == SENT).all()), f"{what}: a resident decode block was written"
+            first_pass = False
+        assert _checksum(src_t) == src_sum, "the prefill pool was written"
+    finally:
+        for s in sessions:
+            s.close()
+    del src_t, pools, buf_t, sessions, stage
     torch.cuda.empty_cache()
 
 
@@ -129,7 +194,7 @@ def test_config2_full_size_same_layout_every_request(oracle):
 
 
 def test_config2_full_size_layer_major_both_sides(oracle):
-    run_fullsize(oracle, W.make_config(2, src_layout=W.LAYER_MAJOR), n_sample=3, seed=22)
+    run_fullsize(oracle, W.make_config(2, src_layout=W.LAYER_MAJOR), n_sample=0, seed=22, group=8)
 
 
 def test_config3_full_size_reblocking_every_request(oracle):
@@ -139,9 +204,9 @@ def test_config3_full_size_reblocking_every_request(oracle):
 def test_config4_full_size_70b_fragmented(oracle):
     w = W.make_config(4)
     assert w.src.num_elems() > 2 ** 32          # offsets beyond 32 bits
-    run_fullsize(oracle, w, n_sample=2, seed=4)
+    run_fullsize(oracle, w, n_sample=0, seed=4, group=2)
 
 
 @pytest.mark.parametrize("src_block", [16, 256])
 def test_config5_full_size_skip_mask(oracle, src_block):
-    run_fullsize(oracle, W.make_config(5, src_block=src_block), n_sample=8, seed=5 + src_block)
+    run_fullsize(oracle, W.make_config(5, src_block=src_block), n_sample=0, seed=5 + src_block, group=16)
