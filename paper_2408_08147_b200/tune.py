@@ -21,6 +21,8 @@ GRIDS = {
                   lc_fastest=[0]),
     "wide": dict(threads=[256, 512, 1024], unroll=[1, 2, 4], ctas_per_sm=[1, 2, 4],
                  tile_bytes=[16384, 32768, 65536, 131072], lc_fastest=[0, 1]),
+    "order": dict(threads=[0], unroll=[0], ctas_per_sm=[2], tile_bytes=[32768, 131072],
+                  lc_fastest=[0, 1], chunked=[0, 1]),
     "bulk": dict(variant=[1, 2], tile_bytes=[8192, 16384, 32768], stages=[2, 3, 4], ctas_per_sm=[2, 3, 4, 6, 8],
                  lc_fastest=[0]),
 }
