@@ -466,7 +466,7 @@ def main_arm(args):
                       "l2": "inputs exceed L2 (pools and buffer are GiB-sized; no flush needed)"
                       if sess.buffer_bytes > (1 << 29) else "L2-resident workload: not an HBM number",
                       "tunables": {k: B.pdkv_tune_get(k) for k in
-                                   ("tile_bytes", "ctas_per_sm", "threads", "unroll", "group_threads", "vec32", "lc_fastest",
+                                   ("tile_bytes", "ctas_per_sm", "threads", "unroll", "group_threads", "vec32", "lc_fastest", "lc_skew",
                                     "variant")}},
            "ops": per_op, "roofline": roofline, "gpu_launches": launches_per_step * args.steps,
            "sanity_check": "ok" if ok else "MISMATCH", "clocks": clk.summary()}

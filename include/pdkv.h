@@ -333,6 +333,19 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream);
  *   "vec32"          1: use 32-byte accesses when rows and bases allow (default 1)
  *   "lc_fastest"     1: consecutive work items walk the (layer, K/V) strips of
  *                    one tile; 0: they walk the tiles of one strip (default 0)
+ *   "lc_skew"        with "lc_fastest" 0, one sweep of the grid moves the same
+ *                    (layer, K/V) strip of every tile.  A skew S (a power of two)
+ *                    lets tile t take strip (s + ((t >> "lc_skew_shift") mod S))
+ *                    mod n_strips in sweep s instead, so that neighbouring blocks
+ *                    are read at different offsets.  0: off; -1 (default):
+ *                    automatic -- 8 for pack / transfer out of a block-major pool
+ *                    whose block stride is 3, 5, 9, 17, ... times a power of two
+ *                    (B200's DRAM handles the same-offset reads of such strides
+ *                    4-9% slower), off otherwise; the register-copy kernels
+ *                    honour it, the bulk-copy variants ignore it
+ *   "lc_skew_shift"  used with an explicit "lc_skew": tiles whose index agrees above
+ *                    this many low bits share a skew (keep the tiles of one prefill
+ *                    block together); chosen automatically with "lc_skew" -1
  *   "chunked"        1: each CTA takes one contiguous run of work items instead
  *                    of every gridDim-th one (default 0)
  *   "debug_bounds"   1: kernels range-check every access and skip bad ones

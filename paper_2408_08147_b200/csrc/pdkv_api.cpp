@@ -235,6 +235,32 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     p.row_bytes = (int32_t)pl->row_bytes;
     p.lc_fastest = (int32_t)pdkv::tunables().lc_fastest;
     p.chunked = (int32_t)pdkv::tunables().chunked;
+    {   // Strip skew (see pdkv_tune "lc_skew").  Automatic: only for calls that read a block-major
+        // pool whose block stride has an odd part with exactly two bits set (3, 5, 9, 17, ... times a
+        // power of two; e.g. 80 layers x 64 tokens x 2 KiB = 5 x 4 MiB).  With such strides the
+        // same-offset strips of many blocks, which one sweep reads at the same time, collide in
+        // DRAM (measured: 4-9% slower than with strides whose odd part is 1, 7, 11 or 13); skewing
+        // the strip by the block's position in the batch spreads them and recovers most of it.
+        // Tiles of one block keep the same skew so that its strip is still read in one piece.
+        int64_t skew = pdkv::tunables().lc_skew, shift = pdkv::tunables().lc_skew_shift;
+        if (skew < 0) {
+            skew = 0;
+            shift = 0;
+            if (op != PDKV_OP_UNPACK && pl->has_src && pl->src.d.layout == PDKV_LAYOUT_BLOCK_MAJOR) {
+                const uint64_t strip = (uint64_t)pl->src.d.block_tokens * (uint64_t)pl->hrow_bytes;
+                uint64_t odd = 2ull * (uint64_t)pl->L * strip;
+                while (odd && !(odd & 1ull)) odd >>= 1;
+                if (__builtin_popcountll(odd) == 2) {
+                    skew = 8;
+                    const uint64_t per_block = pl->max_tile_bytes > 0 ? strip / (uint64_t)pl->max_tile_bytes : 1;
+                    while ((2ull << shift) <= per_block) ++shift;
+                }
+            }
+        }
+        while (skew > 1 && skew > p.n_lc) skew >>= 1;   // a power of two within the strips of this call
+        p.lc_skew = p.lc_fastest ? 0 : (int32_t)skew;
+        p.lc_skew_shift = (int32_t)shift;
+    }
     p.status = pl->dev_status;
     pdkv::LaunchConfig cfg;
     cfg.vec_bytes = pl->vec_bytes;
@@ -805,6 +831,8 @@ int pdkv_tune(const char *key, int64_t value)
     else if (k == "vec32" && (value == 0 || value == 1)) t.vec32 = value;
     else if (k == "lc_fastest" && (value == 0 || value == 1)) t.lc_fastest = value;
     else if (k == "chunked" && (value == 0 || value == 1)) t.chunked = value;
+    else if (k == "lc_skew" && value >= -1 && value <= 1024 && (value < 0 || (value & (value - 1)) == 0)) t.lc_skew = value;
+    else if (k == "lc_skew_shift" && value >= 0 && value <= 20) t.lc_skew_shift = value;
     else if (k == "group_threads" && (value == 0 || (value >= 32 && value <= 1024 && value % 32 == 0))) t.group_threads = value;
     else if (k == "debug_bounds" && (value == 0 || value == 1)) t.debug_bounds = value;
     else if (k == "debug_shrink" && value >= 0) t.debug_shrink = value;
@@ -828,6 +856,8 @@ int pdkv_tune_get(const char *key, int64_t *value)
     else if (k == "vec32") *value = t.vec32;
     else if (k == "lc_fastest") *value = t.lc_fastest;
     else if (k == "chunked") *value = t.chunked;
+    else if (k == "lc_skew") *value = t.lc_skew;
+    else if (k == "lc_skew_shift") *value = t.lc_skew_shift;
     else if (k == "group_threads") *value = t.group_threads;
     else if (k == "debug_bounds") *value = t.debug_bounds;
     else if (k == "debug_shrink") *value = t.debug_shrink;

@@ -40,6 +40,8 @@ struct CopyParams {
     int32_t row_bytes;   // D * E
     int32_t lc_fastest;
     int32_t chunked;     // 1: each group takes one contiguous run of work items
+    int32_t lc_skew;       // power of two <= n_lc, or <= 1 for none: tile t works on strip (s + ((t >> shift) & (skew-1))) mod n_lc in sweep s
+    int32_t lc_skew_shift;
     int32_t group_threads;  // threads that cooperate on one work item (set by the launcher)
     unsigned long long *status;  // [0] != 0: an access was refused; [1] offending offset
 };
@@ -98,6 +100,8 @@ struct Tunables {
     std::atomic<int64_t> lc_fastest{0};
     std::atomic<int64_t> group_threads{0};   // 0: sized from the plan's mean tile
     std::atomic<int64_t> chunked{0};
+    std::atomic<int64_t> lc_skew{-1};   // -1: chosen per call from the prefill pool's block stride
+    std::atomic<int64_t> lc_skew_shift{0};
     std::atomic<int64_t> debug_bounds{0};
     std::atomic<int64_t> debug_shrink{0};   // with debug_bounds: treat the last N bytes of each side as out of range
     std::atomic<int64_t> variant{0};

@@ -143,6 +143,10 @@ copy_tiles_kernel(const CopyParams p)
             lci = (int32_t)(x / p.n_tiles);
             ti = (int32_t)(x - (int64_t)lci * p.n_tiles);
         }
+        if (p.lc_skew > 1) {   // neighbouring tiles take different strips in the same sweep
+            lci += (ti >> p.lc_skew_shift) & (p.lc_skew - 1);
+            if (lci >= p.n_lc) lci -= p.n_lc;
+        }
     };
     // The next item's tile record is fetched while the current one is being
     // copied, so its latency is off the critical path between two tiles.

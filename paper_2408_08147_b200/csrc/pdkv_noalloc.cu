@@ -103,6 +103,8 @@ extern "C" int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
         p.row_bytes = row_bytes;
         p.lc_fastest = (int32_t)t.lc_fastest;
         p.chunked = (int32_t)t.chunked;
+        p.lc_skew = 0;
+        p.lc_skew_shift = 0;
         p.status = reinterpret_cast<unsigned long long *>(slot.scratch);
         pdkv::LaunchConfig cfg;
         cfg.vec_bytes = vec_bytes;

@@ -23,10 +23,12 @@ GRIDS = {
                  tile_bytes=[16384, 32768, 65536, 131072], lc_fastest=[0, 1]),
     "order": dict(threads=[0], unroll=[0], ctas_per_sm=[2], tile_bytes=[32768, 131072],
                   lc_fastest=[0, 1], chunked=[0, 1]),
+    "skew": dict(threads=[0], unroll=[0], ctas_per_sm=[2], tile_bytes=[32768], lc_skew=[-1, 0, 4, 8, 16, 32],
+                 lc_skew_shift=[0, 1, 2, 3]),
     "bulk": dict(variant=[1, 2], tile_bytes=[8192, 16384, 32768], stages=[2, 3, 4], ctas_per_sm=[2, 3, 4, 6, 8],
                  lc_fastest=[0]),
 }
-RESET = dict(variant=0, threads=0, unroll=0, group_threads=0, ctas_per_sm=2, tile_bytes=32768, lc_fastest=0,
+RESET = dict(variant=0, threads=0, unroll=0, group_threads=0, ctas_per_sm=2, tile_bytes=32768, lc_fastest=0, lc_skew=-1, lc_skew_shift=0,
              chunked=0, stages=3, max_ctas=0)
 
 

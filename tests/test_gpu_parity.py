@@ -25,6 +25,8 @@ def _gpu_lib():
     B.pdkv_tune("debug_bounds", 0)
     B.pdkv_tune("tile_bytes", 32768)
     B.pdkv_tune("lc_fastest", 0)
+    B.pdkv_tune("lc_skew", -1)
+    B.pdkv_tune("lc_skew_shift", 0)
     B.pdkv_tune("variant", 0)
     B.pdkv_tune("stages", 3)
 
@@ -112,16 +114,28 @@ def test_scaled_configs(oracle, idx, kw):
     check_all_ops(oracle, w)
 
 
-@pytest.mark.parametrize("tile_bytes,lc_fastest", [(2048, 1), (16384, 0), (1 << 20, 1)])
-def test_tile_size_and_work_order_do_not_change_the_result(oracle, tile_bytes, lc_fastest):
+@pytest.mark.parametrize("tile_bytes,lc_fastest,lc_skew,shift", [(2048, 1, -1, 0), (16384, 0, -1, 0), (1 << 20, 1, 0, 0),
+                                                                 (32768, 0, 8, 2), (4096, 0, 4, 0), (8192, 0, 1024, 3),
+                                                                 (32768, 0, 0, 0)])
+def test_tile_size_and_work_order_do_not_change_the_result(oracle, tile_bytes, lc_fastest, lc_skew, shift):
+    """Tile size, sweep order and strip skew (explicit, automatic = -1, off) only
+    reorder the work.  The 5- and 3-layer cases have block strides of 5 and 3 times a
+    power of two, for which the automatic skew switches itself on; a skew larger than
+    the strips of a call (1024, or 8 on a one-layer range) is cut down to fit."""
     B.pdkv_tune("tile_bytes", tile_bytes)
     B.pdkv_tune("lc_fastest", lc_fastest)
+    B.pdkv_tune("lc_skew", lc_skew)
+    B.pdkv_tune("lc_skew_shift", shift)
     try:
         check_all_ops(oracle, W.make_config(3, num_layers=2, n_req=8, max_len=1200))
         check_all_ops(oracle, W.make_config(5, num_layers=1, n_req=30, src_block=32))
+        check_all_ops(oracle, W.make_config(4, num_layers=5, n_req=3, max_len=500))
+        check_all_ops(oracle, W.make_config(4, num_layers=3, n_req=3, max_len=500), layers=(1, 2))
     finally:
         B.pdkv_tune("tile_bytes", 32768)
         B.pdkv_tune("lc_fastest", 0)
+        B.pdkv_tune("lc_skew", -1)
+        B.pdkv_tune("lc_skew_shift", 0)
 
 
 @pytest.mark.parametrize("variant", [1, 2])
