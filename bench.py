@@ -37,9 +37,9 @@ KERNEL_SOURCE = os.path.join(ROOT, "paper_2408_08147_b200", "csrc", "pdkv_kernel
 # Captured on a 1/8-size case (4 of 32 requests; profiles/copy_tiles_kernel_config2_small_ncu_full.md)
 # and scaled by 8: traffic is proportional to the tokens moved (read 1.0738 GB + write 1.031 GB
 # per 2.1475 GB algorithmic).
-NCU_TRAFFIC: dict = {(2, "pack"): 8 * (1.073880e9 + 1.027572e9), (2, "unpack"): 8 * (1.073865e9 + 1.030411e9),
-                     (2, "fused"): 8 * (1.073906e9 + 1.029486e9)}
-NCU_KERNEL_SHA = "f142536d764dccc3"
+NCU_TRAFFIC: dict = {(2, "pack"): 8 * (1.073864e9 + 1.027792e9), (2, "unpack"): 8 * (1.074102e9 + 1.030286e9),
+                     (2, "fused"): 8 * (1.073851e9 + 1.029149e9)}
+NCU_KERNEL_SHA = "8e42ae40e9fe7366"
 
 
 def log(*a):
