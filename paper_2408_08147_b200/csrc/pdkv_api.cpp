@@ -132,6 +132,18 @@ void build_tiles(pdkv_plan &pl, int op, const pdkv_batch_desc &b, int64_t cap_to
     const int64_t G = pl.G;
     std::vector<Tile> &out = pl.tiles[op];
     const bool want_groups = op == PDKV_OP_TRANSFER;
+    {   // upper bound on the tiles of this list, so that the vectors grow once
+        size_t bound = 0;
+        for (int32_t r = 0; r < pl.n_req; ++r) {
+            const int64_t len = b.seq_len[r];
+            bound += (size_t)(len / cap_tok + 2);
+            if (use_src) bound += (size_t)(len / Bp + 1);
+            if (use_dst) bound += (size_t)(len / Bd + 1 + Bd / cap_tok + 1);
+            if (b.dst_skip) bound += (size_t)(len / G + 1);
+        }
+        out.reserve(bound);
+        if (want_groups) pl.groups.reserve(bound);
+    }
     const bool same_blocks = want_groups && pl.src.d.layout == PDKV_LAYOUT_BLOCK_MAJOR &&
                              pl.dst.d.layout == PDKV_LAYOUT_BLOCK_MAJOR && Bp == Bd;
     for (int32_t r = 0; r < pl.n_req; ++r) {
