@@ -652,6 +652,10 @@ def overlap_arm(args):
                                                   "max_ctas": 64}),
              ("register copy on at most 32 SMs", {"variant": 0, "ctas_per_sm": 1, "threads": 1024, "unroll": 1,
                                                   "max_ctas": 32}),
+             ("register copy, one warp per CTA (32 threads x 8 accesses), 4 CTAs/SM",
+              {"variant": 0, "ctas_per_sm": 4, "threads": 32, "unroll": 8, "group_threads": 32}),
+             ("register copy, two warps per CTA (64 threads x 4 accesses), 8 CTAs/SM",
+              {"variant": 0, "ctas_per_sm": 8, "threads": 64, "unroll": 4, "group_threads": 64}),
              ("bulk copy (TMA), 8 KiB tiles x 2 stages x 8 CTAs/SM",
               {"variant": 1, "tile_bytes": 8192, "stages": 2, "ctas_per_sm": 8}),
              ("bulk copy with tiled TMA loads, 16 KiB tiles x 4 stages x 3 CTAs/SM",
@@ -659,7 +663,7 @@ def overlap_arm(args):
              ("bulk copy with tiled TMA loads, 16 KiB tiles x 2 stages x 2 CTAs/SM",
               {"variant": 2, "tile_bytes": 16384, "stages": 2, "ctas_per_sm": 2})]
     defaults = {k: B.pdkv_tune_get(k) for k in ("variant", "ctas_per_sm", "threads", "unroll", "tile_bytes", "stages",
-                                                "max_ctas")}
+                                                "max_ctas", "group_threads")}
     t_compute = timed(compute_only, args.steps)
     for name, tune in modes:
         for k, v in {**defaults, **tune}.items():
