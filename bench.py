@@ -758,6 +758,85 @@ def retrieval_arm(args):
     print(json.dumps(out), flush=True)
 
 
+def p2d_arm(args):
+    """Prefill-to-decode transfer between two ranks on two GPUs (Sec. 3.5; launch with
+    torchrun --nproc-per-node 2): rank 0 holds the prefill pool and packs, the buffer
+    crosses NVLink in one NCCL send / recv, rank 1 unpacks.  Times the block-free
+    transfer against the same bytes sent one prefill block's worth at a time."""
+    import torch
+
+    from paper_2408_08147_b200 import binding as B
+    from paper_2408_08147_b200 import p2d
+    from paper_2408_08147_b200 import workloads as W
+
+    rank, local, world = dist_env()
+    if world != 2:
+        if rank == 0:
+            print(json.dumps({"mode": "p2d", "unavailable": "needs exactly two ranks, one GPU each"}), flush=True)
+        return
+    B.lib()
+    host = args.p2d_host_buffers      # buffer in pinned host memory, gloo carries it; the ranks may share a GPU
+    local = local % torch.cuda.device_count() if host else local
+    torch.cuda.set_device(local)
+    dist_init("gloo" if host else "nccl")
+    dev = torch.device("cuda", local)
+    meta_dev = "cpu" if host else dev
+    kw = {"n_req": args.n_req} if args.n_req else {}
+    if args.num_layers:
+        kw["num_layers"] = args.num_layers
+    w = W.make_config(args.config, **kw)
+    b = w.batch
+    if rank == 0:
+        pool_t = torch.empty(w.src.num_bytes(), dtype=torch.uint8, device=dev)
+        W.fill_pool_torch(pool_t, w.seed)
+    else:
+        pool_t = torch.zeros(w.dst.num_bytes(), dtype=torch.uint8, device=dev)
+    torch.cuda.synchronize()
+    cache = {}
+
+    def buffer(n):                      # one buffer per rank, reused across repetitions
+        if cache.get("n", 0) < n:
+            cache["t"] = torch.empty(n, dtype=torch.uint8, pin_memory=True) if host else \
+                torch.empty(n, dtype=torch.uint8, device=dev)
+            cache["n"] = n
+        return cache["t"][:n]
+
+    block_bytes = w.src.num_bytes() // w.src.num_blocks
+    results = {}
+    for name, chunk in (("whole buffer", 0), ("one prefill block per message", block_bytes)):
+        times, nbytes = [], 0
+        for it in range(args.warmup + args.steps):
+            barrier()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            if rank == 0:
+                nbytes, sess, _ = p2d.send_kv(b.seq_len, p2d.gpu_sender(w.src, pool_t, b.src_tbl_off, b.src_tbl, b.seq_len),
+                                              buffer, peer=1, device=meta_dev, chunk_bytes=chunk)
+            else:
+                nbytes, sess, _ = p2d.recv_kv(b.dst_tbl_off, b.dst_skip, w.dst.block_tokens,
+                                              p2d.gpu_receiver(w.dst, pool_t, b.dst_tbl_off, b.dst_tbl, b.dst_skip),
+                                              buffer, peer=0, device=meta_dev, chunk_bytes=chunk)
+            torch.cuda.synchronize()
+            dt = (time.perf_counter() - t0) * 1e3
+            sess.close()
+            ms, _ = reduce_step_time(dt, 0.0, meta_dev)
+            if it >= args.warmup:
+                times.append(ms)
+        results[name] = {"ms": statistics.fmean(times), "ms_best": min(times), "buffer_bytes": nbytes,
+                         "link_GBps": nbytes / (statistics.fmean(times) * 1e-3) / 1e9,
+                         "messages": max(1, -(-nbytes // chunk)) if chunk else 1}
+    if rank == 0:
+        a, c = results["whole buffer"]["ms"], results["one prefill block per message"]["ms"]
+        print(json.dumps({"mode": "p2d", "config": {"workload": workload_name(w)}, "variants": results,
+                          "time_saved_by_block_free": 1.0 - a / c,
+                          "transport": "gloo, pinned host buffers" if host else "NCCL send/recv between two GPUs",
+                          "includes": "meta exchange, plan, pack, send/recv, unpack; wall clock, max over ranks"}),
+              flush=True)
+    import torch.distributed as dist
+
+    dist.destroy_process_group()
+
+
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -780,6 +859,9 @@ def parse():
     ap.add_argument("--overlap", action="store_true", help="per-layer transfer overlapped with a compute stand-in")
     ap.add_argument("--retrieval", action="store_true", help="request groups through the asynchronous retrieval queue")
     ap.add_argument("--retrieval-groups", type=int, default=8)
+    ap.add_argument("--p2d", action="store_true", help="two ranks, two GPUs: pack -> one NCCL send/recv -> unpack")
+    ap.add_argument("--p2d-host-buffers", action="store_true",
+                    help="with --p2d: contiguous buffer in pinned host memory, gloo transport; the two ranks may share one GPU")
     ap.add_argument("--gemm-n", type=int, default=4096)
     ap.add_argument("--side-priority", type=int, default=1, help="1: transfer stream has high priority")
     ap.add_argument("--no-blockwise", action="store_true")
@@ -793,6 +875,8 @@ if __name__ == "__main__":
         overlap_arm(a)
     elif a.retrieval:
         retrieval_arm(a)
+    elif a.p2d:
+        p2d_arm(a)
     elif a.impl == "reference":
         reference_arm(a)
     else:

@@ -92,6 +92,10 @@ class TransferSession:
     def status(self, stream: Optional[int] = None) -> None:
         B.pdkv_plan_status(self.plan, self.stream if stream is None else stream)
 
+    def synchronize(self, stream: Optional[int] = None) -> None:
+        """Wait for the session's stream (and raise if a kernel reported an error)."""
+        self.status(stream)
+
     def traffic(self, op: int):
         return B.pdkv_plan_traffic(self.plan, op)
 
