@@ -338,10 +338,10 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream);
  *                    lets tile t take strip (s + ((t >> "lc_skew_shift") mod S))
  *                    mod n_strips in sweep s instead, so that neighbouring blocks
  *                    are read at different offsets.  0: off; -1 (default):
- *                    automatic -- 8 for calls that read (else write) a block-major
- *                    pool whose block stride is 3, 5, 9, 17, ... times a power of
- *                    two (B200's DRAM handles same-offset accesses at such strides
- *                    2-9% slower), off otherwise; the register-copy kernels
+ *                    automatic -- 16 for calls that read (else write) a block-major
+ *                    pool whose block stride is a power of two times a multiple of
+ *                    3, 5 or 17 (B200's DRAM handles same-offset accesses at such strides
+ *                    2-12% slower), off otherwise; the register-copy kernels
  *                    honour it, the bulk-copy variants ignore it
  *   "lc_skew_shift"  used with an explicit "lc_skew": tiles whose index agrees above
  *                    this many low bits share a skew (keep the tiles of one prefill

@@ -248,13 +248,13 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     p.lc_fastest = (int32_t)pdkv::tunables().lc_fastest;
     p.chunked = (int32_t)pdkv::tunables().chunked;
     {   // Strip skew (see pdkv_tune "lc_skew").  Automatic: only for calls that read (or, failing
-        // that, write) a block-major pool whose block stride has an odd part with exactly two bits
-        // set (3, 5, 9, 17, ... times a power of two; e.g. 80 layers x 64 tokens x 2 KiB = 5 x 4 MiB).
-        // With such strides the same-offset strips of many blocks, which one sweep touches at the
-        // same time, collide in DRAM (measured: reads 4-9% and writes 2% slower than with strides
-        // whose odd part is 1, 7, 11 or 13); skewing the strip by the block's position in the batch
-        // spreads them and recovers most of it.  Tiles of one block keep the same skew so that
-        // its strip is still moved in one piece.
+        // that, write) a block-major pool whose block stride, stripped of its factors of two, is
+        // divisible by 3, 5 or 17 (e.g. 80 layers x 64 tokens x 2 KiB = 5 x 4 MiB).  With such
+        // strides the same-offset strips of many blocks, which one sweep touches at the same
+        // time, collide in DRAM (measured on 37 strides: reads 4-12% and writes 2% slower, every
+        // odd part sharing a factor with 255 and no other); skewing the strip by the block's
+        // position in the batch spreads them and recovers most of it.  Tiles of one block keep
+        // the same skew so that its strip is still moved in one piece.
         int64_t skew = pdkv::tunables().lc_skew, shift = pdkv::tunables().lc_skew_shift;
         if (skew < 0) {
             skew = 0;
@@ -264,8 +264,8 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
                 const uint64_t strip = (uint64_t)pool.d.block_tokens * (uint64_t)pl->hrow_bytes;
                 uint64_t odd = 2ull * (uint64_t)pl->L * strip;
                 while (odd && !(odd & 1ull)) odd >>= 1;
-                if (__builtin_popcountll(odd) != 2) return;
-                skew = 8;
+                if (odd % 3 && odd % 5 && odd % 17) return;
+                skew = 16;
                 const uint64_t per_block = pl->max_tile_bytes > 0 ? strip / (uint64_t)pl->max_tile_bytes : 1;
                 while ((2ull << shift) <= per_block) ++shift;
             };
