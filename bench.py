@@ -383,6 +383,8 @@ def main_arm(args):
         kw["num_kv_heads"] = args.kv_heads
     if args.num_layers:
         kw["num_layers"] = args.num_layers
+    if args.head_dim:
+        kw["head_dim"] = args.head_dim
     if args.layouts:
         kw["src_layout"], kw["dst_layout"] = ("AB".index(args.layouts[0]), "AB".index(args.layouts[1]))
     w = W.make_config(args.config, **kw)
@@ -847,6 +849,7 @@ def parse():
     ap.add_argument("--src-block", type=int, default=0)
     ap.add_argument("--elem-bytes", type=int, default=0, help="KV element size override (1 = fp8/int8 KV)")
     ap.add_argument("--kv-heads", type=int, default=0, help="KV head count override (1 = MQA)")
+    ap.add_argument("--head-dim", type=int, default=0, help="head dimension override (e.g. 96)")
     ap.add_argument("--n-req", type=int, default=0, help="shrink the batch (profiling captures)")
     ap.add_argument("--num-layers", type=int, default=0, help="shrink the model (profiling captures)")
     ap.add_argument("--layouts", default="", help="two letters, e.g. AB: prefill block-major, decode layer-major")

@@ -156,10 +156,16 @@ void build_tiles(pdkv_plan &pl, int op, const pdkv_batch_desc &b, int64_t cap_to
                 t = std::min(len, (t / G + 1) * G);
                 continue;
             }
-            int64_t end = std::min(len, t + cap_tok);
+            // the run up to the next boundary is cut into equal pieces no longer than the cap,
+            // not into full pieces and a short rest
+            int64_t end = len;
             if (skip) end = std::min(end, (t / G + 1) * G);
             if (use_src) end = std::min(end, (t / Bp + 1) * Bp);
             if (use_dst) end = std::min(end, (t / Bd + 1) * Bd);
+            {
+                const int64_t run = end - t, pieces = (run + cap_tok - 1) / cap_tok;
+                end = t + (run + pieces - 1) / pieces;
+            }
             Tile tl;
             tl.ntok = (int32_t)(end - t);
             tl.n_kept = (int32_t)pl.kept[r];
@@ -196,9 +202,11 @@ void build_tiles(pdkv_plan &pl, int op, const pdkv_batch_desc &b, int64_t cap_to
             const int64_t first_pad = len - (nb - 1) * Bd;
             if (first_pad < Bd && !(skip && skip[nb - 1])) {
                 const int64_t blk = b.dst_tbl[b.dst_tbl_off[r] + nb - 1];
-                for (int64_t tt = first_pad; tt < Bd; tt += cap_tok) {
+                const int64_t pad_pieces = (Bd - first_pad + cap_tok - 1) / cap_tok;
+                const int64_t pad_tok = (Bd - first_pad + pad_pieces - 1) / pad_pieces;
+                for (int64_t tt = first_pad; tt < Bd; tt += pad_tok) {
                     Tile tl;
-                    tl.ntok = (int32_t)std::min(cap_tok, Bd - tt);
+                    tl.ntok = (int32_t)std::min(pad_tok, Bd - tt);
                     tl.n_kept = (int32_t)pl.kept[r];
                     tl.src_off = -1;
                     tl.dst_off = pool_tile_off(pl.dst.d, blk, tt, pl.row_bytes, pl.hrow_bytes);
