@@ -30,16 +30,16 @@ if ROOT not in sys.path:
 METRIC = "KV pack+unpack+fused transfer throughput (algorithmic bytes read+written)"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
-KERNEL_SOURCE = os.path.join(ROOT, "paper_2408_08147_b200", "csrc", "pdkv_kernels.cu")
+KERNEL_SOURCE = os.path.join(ROOT, "paper_2408_08147_b200", "csrc", "pdkv_copy_kernel.cuh")   # device code only
 
 # DRAM traffic per launch from ncu (dram__bytes_read.sum + dram__bytes_write.sum),
 # keyed by (workload, op); valid only while the kernel source hashes to KERNEL_SHA.
 # Captured on a 1/8-size case (4 of 32 requests; profiles/copy_tiles_kernel_config2_small_ncu_full.md)
 # and scaled by 8: traffic is proportional to the tokens moved (read 1.0738 GB + write 1.031 GB
 # per 2.1475 GB algorithmic).
-NCU_TRAFFIC: dict = {(2, "pack"): 8 * (1.073864e9 + 1.027792e9), (2, "unpack"): 8 * (1.074102e9 + 1.030286e9),
-                     (2, "fused"): 8 * (1.073851e9 + 1.029149e9)}
-NCU_KERNEL_SHA = "8e42ae40e9fe7366"
+NCU_TRAFFIC: dict = {(2, "pack"): 8 * (1.074156e9 + 1.028752e9), (2, "unpack"): 8 * (1.073918e9 + 1.030543e9),
+                     (2, "fused"): 8 * (1.074030e9 + 1.029745e9)}
+NCU_KERNEL_SHA = "7e27088e22471cf0"
 
 
 def log(*a):
