@@ -402,6 +402,10 @@ def main_arm(args):
     ops = [("pack", B.PDKV_OP_PACK, lambda: sess.pack(buf_t)),
            ("unpack", B.PDKV_OP_UNPACK, lambda: sess.unpack(buf_t)),
            ("fused", B.PDKV_OP_TRANSFER, lambda: sess.transfer())]
+    tuned = None
+    if args.autotune:
+        tuned = {str(k): v for k, v in sess.autotune(buf_t).items()}
+        torch.cuda.synchronize()
     traffic = {name: sum(sess.traffic(op)) for name, op, _ in ops}
     step_bytes = sum(traffic.values())
     launches_per_step = sum(sess.launches(op) for _, op, _ in ops)
@@ -465,6 +469,7 @@ def main_arm(args):
                       "step": "pdkv_pack + pdkv_unpack + pdkv_transfer, all layers",
                       "payload_bytes": sess.buffer_bytes, "step_bytes": step_bytes,
                       "plan_create_destroy_ms": statistics.median(plan_ms),
+                      "autotuned_shapes (threads, unroll, CTAs/SM per op; zeros = built-in)": tuned,
                       "l2": "inputs exceed L2 (pools and buffer are GiB-sized; no flush needed)"
                       if sess.buffer_bytes > (1 << 29) else "L2-resident workload: not an HBM number",
                       "tunables": {k: B.pdkv_tune_get(k) for k in
@@ -868,6 +873,7 @@ def parse():
     ap.add_argument("--gemm-n", type=int, default=4096)
     ap.add_argument("--side-priority", type=int, default=1, help="1: transfer stream has high priority")
     ap.add_argument("--no-blockwise", action="store_true")
+    ap.add_argument("--autotune", action="store_true", help="pdkv_plan_autotune before the timed steps (not the default run)")
     return ap.parse_args()
 
 

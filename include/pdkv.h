@@ -159,6 +159,36 @@ int pdkv_plan_create_in(const pdkv_pool *src, const pdkv_pool *dst,
  * the plan has completed (its kernels read the tile lists). */
 int pdkv_plan_destroy(pdkv_plan *plan);
 
+/* Optional: find the launch shape (threads per CTA, accesses in flight per thread,
+ * CTAs per SM) of each operation by timing it on this batch.  The built-in
+ * choice is tuned for Llama-shaped geometries (32 KiB tiles of 256-byte rows);
+ * other head sizes, head counts or block sizes can run several percent -- for
+ * 160-byte rows up to 30% -- faster with a shape that covers one of their tiles
+ * in exactly one or two passes.  About ten candidate shapes are launched a few
+ * times each over some or all layers of the batch, for pack and unpack (only
+ * if `buf` is given: device, at least pdkv_plan_buffer() bytes) and for
+ * transfer; a shape replaces the built-in one only if it is more than 1.5%
+ * faster.  The operations are the real ones: afterwards `buf` holds the packed
+ * layers and the decode pool the transferred layers that were used for timing
+ * (with an unpack-only plan `buf` must already hold a packed batch).  The
+ * call synchronises `stream` repeatedly; it is meant for set-up time, once per
+ * geometry: the result is kept in the plan and, unless "autotune_reuse" is 0,
+ * remembered for every later plan of the process with the same pool
+ * geometries and tile sizes.  Explicit "threads" / "unroll" tunables override
+ * it.  Plans with small tiles (under 8 KiB) are left alone.  (No counterpart in
+ * the paper.)  pdkv_plan_shape() reports what a plan uses (zeros: built-in).
+ * Errors: INVALID_ARG, BUFFER_TOO_SMALL, CUDA. */
+int pdkv_plan_autotune(pdkv_plan *plan, void *buf, size_t buf_bytes, void *stream);
+int pdkv_plan_shape(const pdkv_plan *plan, int op, int32_t *threads, int32_t *unroll,
+                    int32_t *ctas_per_sm);
+/* Pin the launch shape of one operation of this plan by hand (threads: multiple of
+ * 32 up to 1024, clamped to what the register budget allows; unroll: 1, 2, 4 or 8;
+ * ctas_per_sm: 1..32); all three zero returns to the built-in choice.  Not
+ * thread-safe against launches that use the plan at the same time.
+ * Errors: INVALID_ARG. */
+int pdkv_plan_set_shape(pdkv_plan *plan, int op, int32_t threads, int32_t unroll,
+                        int32_t ctas_per_sm);
+
 /* Size of the contiguous buffer in bytes and, optionally, the host array of
  * n_req+1 request offsets off_r (owned by the plan, valid until destroy). */
 int pdkv_plan_buffer(const pdkv_plan *plan, size_t *total_bytes,
@@ -361,6 +391,8 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream);
  *                    geometry meets the TMA rules
  *   "stages"         variant 1: shared-memory stages per CTA, 2..16 (default 3);
  *                    stages x "tile_bytes" must fit in 220 KiB
+ *   "autotune_reuse" 1 (default): a new plan starts with the shapes that an earlier
+ *                    pdkv_plan_autotune() found for the same geometry
  *   "dry_run"        1: pdkv_plan_create builds host-only plans (no CUDA call is
  *                    made; the plan can be inspected but not launched)
  * Unknown keys or out-of-range values give INVALID_ARG. */

@@ -43,6 +43,7 @@ EXPORTS = (
     "pdkv_plan_status", "pdkv_upload_blocks", "pdkv_download_blocks", "pdkv_plan_block_bytes",
     "pdkv_queue_create", "pdkv_queue_submit", "pdkv_queue_poll", "pdkv_queue_wait", "pdkv_queue_release",
     "pdkv_queue_stats", "pdkv_queue_destroy", "pdkv_tune", "pdkv_tune_get", "pdkv_strerror",
+    "pdkv_plan_autotune", "pdkv_plan_shape", "pdkv_plan_set_shape",
 )
 
 
@@ -201,6 +202,22 @@ def pdkv_plan_create_in(src_pool: Optional[int], dst_pool: Optional[int], skip_g
         err.needed_bytes = int(need.value)
         raise err
     return out.value, int(need.value)
+
+
+def pdkv_plan_autotune(plan: int, buf_ptr: int = 0, buf_bytes: int = 0, stream: int = 0) -> None:
+    _check(lib().pdkv_plan_autotune(C.c_void_p(plan), C.c_void_p(buf_ptr), C.c_size_t(buf_bytes),
+                                    C.c_void_p(stream)), "pdkv_plan_autotune")
+
+
+def pdkv_plan_shape(plan: int, op: int):
+    """(threads, unroll, ctas_per_sm) the plan uses for ``op``; zeros = the built-in choice."""
+    t, u, c = C.c_int32(), C.c_int32(), C.c_int32()
+    _check(lib().pdkv_plan_shape(C.c_void_p(plan), op, C.byref(t), C.byref(u), C.byref(c)), "pdkv_plan_shape")
+    return int(t.value), int(u.value), int(c.value)
+
+
+def pdkv_plan_set_shape(plan: int, op: int, threads: int, unroll: int, ctas_per_sm: int) -> None:
+    _check(lib().pdkv_plan_set_shape(C.c_void_p(plan), op, threads, unroll, ctas_per_sm), "pdkv_plan_set_shape")
 
 
 def pdkv_plan_destroy(plan: int) -> None:

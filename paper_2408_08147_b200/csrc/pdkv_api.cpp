@@ -4,8 +4,11 @@
 // precision), cuts the batch into tiles and uploads the tile lists once.  This
 // is the single-GPU counterpart of the meta exchange that precedes a transfer.
 #include <algorithm>
+#include <array>
 #include <cstdio>
 #include <cstring>
+#include <map>
+#include <mutex>
 #include <new>
 #include <string>
 
@@ -81,7 +84,10 @@ struct pdkv_plan {
     int64_t max_tile_bytes = 0;
     int64_t mean_tile_bytes[3] = {0, 0, 0};   // per operation, over its tile list
     int sm_count = 1;
-    int lc_fastest = 1;
+    // launch shape found by pdkv_plan_autotune() for each operation; threads == 0: not tuned
+    struct Shape {
+        int threads = 0, unroll = 0, ctas_per_sm = 0;
+    } shape[3];
 };
 
 namespace {
@@ -308,9 +314,17 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
         const bool flat = src.head_stride == row && src.tok_stride == hrow && dst.head_stride == row &&
                           dst.tok_stride == hrow;
         const bool small = pl->mean_tile_bytes[op] < 24 * 1024;
+        const pdkv_plan::Shape &tuned = pl->shape[op];
+        const bool use_tuned = tuned.threads > 0 && cfg.unroll == 0 && cfg.threads == 0;
+        if (use_tuned) {   // found by pdkv_plan_autotune(): the whole CTA works on one tile
+            cfg.threads = tuned.threads;
+            cfg.unroll = tuned.unroll;
+            cfg.ctas_per_sm = tuned.ctas_per_sm;
+        }
         if (cfg.unroll == 0) cfg.unroll = (flat || small) ? 1 : 4;
         if (cfg.threads == 0) cfg.threads = (flat || small) ? 512 : 256;
         cfg.group_threads = (int)pdkv::tunables().group_threads;
+        if (use_tuned && cfg.group_threads == 0) cfg.group_threads = cfg.threads;
         if (cfg.group_threads == 0) {
             const int64_t vecs = std::max<int64_t>(1, pl->mean_tile_bytes[op] / cfg.vec_bytes);
             const int64_t want = vecs / ((flat || small) ? 2 : cfg.unroll);
@@ -342,6 +356,31 @@ bool ranges_overlap(const void *a, size_t a_bytes, const void *b, size_t b_bytes
     const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
     return a_bytes && b_bytes && a0 < b0 + b_bytes && b0 < a0 + a_bytes;
 }
+
+}  // namespace
+
+namespace {
+
+// Shapes found by pdkv_plan_autotune(), remembered per geometry for later plans of the process.
+struct ShapeKey {
+    int32_t v[12];
+    bool operator<(const ShapeKey &o) const { return std::lexicographical_compare(v, v + 12, o.v, o.v + 12); }
+};
+
+ShapeKey shape_key(const pdkv_plan *pl)
+{
+    ShapeKey k{};
+    const pdkv_pool_desc *s = pl->has_src ? &pl->src.d : nullptr, *d = pl->has_dst ? &pl->dst.d : nullptr;
+    k.v[0] = pl->L; k.v[1] = pl->H; k.v[2] = pl->D; k.v[3] = pl->E;
+    k.v[4] = s ? s->layout : -1; k.v[5] = s ? s->block_tokens : 0;
+    k.v[6] = d ? d->layout : -1; k.v[7] = d ? d->block_tokens : 0;
+    k.v[8] = (int32_t)std::min<int64_t>(pl->max_tile_bytes, INT32_MAX);
+    for (int op = 0; op < 3; ++op) k.v[9 + op] = (int32_t)std::min<int64_t>(pl->mean_tile_bytes[op] >> 10, INT32_MAX);
+    return k;
+}
+
+std::mutex g_shapes_mutex;
+std::map<ShapeKey, std::array<pdkv_plan::Shape, 3>> g_shapes;
 
 }  // namespace
 
@@ -467,7 +506,6 @@ int pdkv_plan_create_in(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip
         pl->row_bytes = (int64_t)pl->D * pl->E;
         pl->hrow_bytes = pl->row_bytes * pl->H;
         pl->n_req = batch->n_req;
-        pl->lc_fastest = (int)pdkv::tunables().lc_fastest;
 
         int rc;
         if (src && (rc = check_table(batch->src_tbl_off, batch->src_tbl, batch->n_req, batch->seq_len,
@@ -584,6 +622,13 @@ int pdkv_plan_create_in(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip
             pl->mean_tile_bytes[op] = pl->tiles[op].empty() ? 0 : sum / (int64_t)pl->tiles[op].size();
         }
 
+        if (pdkv::tunables().autotune_reuse) {   // shapes an earlier pdkv_plan_autotune() found for this geometry
+            std::lock_guard<std::mutex> lock(g_shapes_mutex);
+            auto it = g_shapes.find(shape_key(pl));
+            if (it != g_shapes.end())
+                for (int op = 0; op < 3; ++op) pl->shape[op] = it->second[(size_t)op];
+        }
+
         // device bytes of the plan: [status words][pack tiles][unpack tiles][transfer tiles]
         const size_t head = 256;
         size_t total = head;
@@ -634,6 +679,125 @@ int pdkv_plan_create_in(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip
     } catch (const std::bad_alloc &) {
         return PDKV_ERR_NOMEM;
     }
+}
+
+int pdkv_plan_autotune(pdkv_plan *plan, void *buf, size_t buf_bytes, void *stream)
+{
+    if (!plan || !plan->dev_mem) return PDKV_ERR_INVALID_ARG;
+    const bool with_buf = buf != nullptr;
+    if (with_buf && buf_bytes < plan->payload_bytes) return PDKV_ERR_BUFFER_TOO_SMALL;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    cudaError_t e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    if (e != cudaSuccess) {
+        if (e0) cudaEventDestroy(e0);
+        return cuda_fail(e, "cudaEventCreate");
+    }
+    // enough layers for a launch of a few hundred MiB, all of them for small batches
+    int layers = plan->L;
+    const uint64_t want_bytes = 1ull << 30;
+    if (plan->payload_bytes > want_bytes)
+        layers = (int)std::max<uint64_t>(2, std::min<uint64_t>((uint64_t)plan->L, (uint64_t)plan->L * want_bytes / plan->payload_bytes));
+    layers = std::min(layers, (int)plan->L);
+
+    int rc = PDKV_OK;
+    auto run = [&](int op) -> int {
+        if (op == PDKV_OP_PACK) return pdkv_pack(plan, buf, buf_bytes, 0, layers, stream);
+        if (op == PDKV_OP_UNPACK) return pdkv_unpack(plan, buf, buf_bytes, 0, layers, stream);
+        return pdkv_transfer(plan, 0, layers, stream);
+    };
+    auto time_ms = [&](int op, float *ms) -> int {
+        const int reps = 3;
+        int r = run(op);   // warm-up, and the first touch of a new instantiation
+        if (r != PDKV_OK) return r;
+        cudaError_t ce = cudaEventRecord(e0, st);
+        for (int i = 0; i < reps && r == PDKV_OK; ++i) r = run(op);
+        if (r != PDKV_OK) return r;
+        if (ce == cudaSuccess) ce = cudaEventRecord(e1, st);
+        if (ce == cudaSuccess) ce = cudaEventSynchronize(e1);
+        if (ce == cudaSuccess) ce = cudaEventElapsedTime(ms, e0, e1);
+        if (ce != cudaSuccess) return cuda_fail(ce, "autotune timing");
+        *ms /= reps;
+        return PDKV_OK;
+    };
+    for (int op = 0; op < 3 && rc == PDKV_OK; ++op) {
+        if (plan->tiles[op].empty() || plan->payload_bytes == 0) continue;
+        if (op != PDKV_OP_TRANSFER && !with_buf) continue;
+        if ((op != PDKV_OP_UNPACK && !plan->has_src) || (op != PDKV_OP_PACK && !plan->has_dst)) continue;
+        if (plan->mean_tile_bytes[op] < 8 * 1024) continue;   // small tiles: thread groups, sized automatically
+        const int vec = (plan->vec_bytes == 16 && plan->row_bytes % 32 == 0) ? 32 : plan->vec_bytes;
+        const int64_t nvec = std::max<int64_t>(1, plan->mean_tile_bytes[op] / vec);
+        std::vector<pdkv_plan::Shape> cand;
+        auto add = [&](int64_t threads, int unroll, int ctas) {
+            threads = (threads + 31) / 32 * 32;
+            const int cap = vec * unroll >= 256 ? 256 : (vec * unroll >= 128 ? 512 : 1024);
+            if (threads < 64 || threads > cap) return;
+            for (const auto &c : cand)
+                if (c.threads == threads && c.unroll == unroll && c.ctas_per_sm == ctas) return;
+            pdkv_plan::Shape s;
+            s.threads = (int)threads;
+            s.unroll = unroll;
+            s.ctas_per_sm = ctas;
+            cand.push_back(s);
+        };
+        add(256, 4, 2); add(512, 1, 2); add(512, 2, 2); add(256, 1, 4); add(1024, 1, 1); add(256, 2, 2);
+        add(nvec, 1, 2); add((nvec + 1) / 2, 2, 2); add((nvec + 3) / 4, 4, 2);       // one pass = one tile
+        add((nvec + 1) / 2, 1, 2); add((nvec + 3) / 4, 2, 2);                         // two passes = one tile
+        plan->shape[op] = pdkv_plan::Shape();
+        float best_ms = 0.f;
+        rc = time_ms(op, &best_ms);              // the per-class default is the incumbent
+        pdkv_plan::Shape best;
+        for (size_t i = 0; i < cand.size() && rc == PDKV_OK; ++i) {
+            plan->shape[op] = cand[i];
+            float ms = 0.f;
+            rc = time_ms(op, &ms);
+            if (rc == PDKV_OK && ms < 0.985f * best_ms) {   // a candidate must win by more than the noise
+                best_ms = ms;
+                best = cand[i];
+            }
+        }
+        plan->shape[op] = best;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (rc != PDKV_OK) {
+        for (int op = 0; op < 3; ++op) plan->shape[op] = pdkv_plan::Shape();
+        return rc;
+    }
+    {
+        std::lock_guard<std::mutex> lock(g_shapes_mutex);
+        std::array<pdkv_plan::Shape, 3> all = {plan->shape[0], plan->shape[1], plan->shape[2]};
+        g_shapes[shape_key(plan)] = all;
+    }
+    return PDKV_OK;
+}
+
+int pdkv_plan_set_shape(pdkv_plan *plan, int op, int32_t threads, int32_t unroll, int32_t ctas_per_sm)
+{
+    if (!plan || op < 0 || op > 2) return PDKV_ERR_INVALID_ARG;
+    if (threads == 0 && unroll == 0 && ctas_per_sm == 0) {   // back to the built-in choice
+        plan->shape[op] = pdkv_plan::Shape();
+        return PDKV_OK;
+    }
+    if (threads < 32 || threads > 1024 || threads % 32 || (unroll != 1 && unroll != 2 && unroll != 4 && unroll != 8) ||
+        ctas_per_sm < 1 || ctas_per_sm > 32)
+        return PDKV_ERR_INVALID_ARG;
+    plan->shape[op].threads = threads;
+    plan->shape[op].unroll = unroll;
+    plan->shape[op].ctas_per_sm = ctas_per_sm;
+    return PDKV_OK;
+}
+
+int pdkv_plan_shape(const pdkv_plan *plan, int op, int32_t *threads, int32_t *unroll, int32_t *ctas_per_sm)
+{
+    if (!plan || op < 0 || op > 2) return PDKV_ERR_INVALID_ARG;
+    if (threads) *threads = plan->shape[op].threads;
+    if (unroll) *unroll = plan->shape[op].unroll;
+    if (ctas_per_sm) *ctas_per_sm = plan->shape[op].ctas_per_sm;
+    return PDKV_OK;
 }
 
 int pdkv_plan_destroy(pdkv_plan *plan)
@@ -862,6 +1026,7 @@ int pdkv_tune(const char *key, int64_t value)
     else if (k == "variant" && value >= 0 && value <= 2) t.variant = value;
     else if (k == "stages" && value >= 2 && value <= 16) t.stages = value;
     else if (k == "dry_run" && (value == 0 || value == 1)) t.dry_run = value;
+    else if (k == "autotune_reuse" && (value == 0 || value == 1)) t.autotune_reuse = value;
     else return PDKV_ERR_INVALID_ARG;
     return PDKV_OK;
 }
@@ -887,6 +1052,7 @@ int pdkv_tune_get(const char *key, int64_t *value)
     else if (k == "variant") *value = t.variant;
     else if (k == "stages") *value = t.stages;
     else if (k == "dry_run") *value = t.dry_run;
+    else if (k == "autotune_reuse") *value = t.autotune_reuse;
     else return PDKV_ERR_INVALID_ARG;
     return PDKV_OK;
 }

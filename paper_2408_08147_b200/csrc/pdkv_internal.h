@@ -107,6 +107,7 @@ struct Tunables {
     std::atomic<int64_t> variant{0};
     std::atomic<int64_t> stages{3};
     std::atomic<int64_t> dry_run{0};
+    std::atomic<int64_t> autotune_reuse{1};
 };
 Tunables &tunables();
 

@@ -92,6 +92,14 @@ class TransferSession:
     def status(self, stream: Optional[int] = None) -> None:
         B.pdkv_plan_status(self.plan, self.stream if stream is None else stream)
 
+    def autotune(self, buf_t=None, stream: Optional[int] = None):
+        """Time candidate launch shapes on this batch and keep the fastest per operation
+        (pack and unpack only if ``buf_t`` is given).  Returns the shapes per operation."""
+        B.pdkv_plan_autotune(self.plan, buf_t.data_ptr() if buf_t is not None else 0,
+                             buf_t.numel() * buf_t.element_size() if buf_t is not None else 0,
+                             self.stream if stream is None else stream)
+        return {op: B.pdkv_plan_shape(self.plan, op) for op in (B.PDKV_OP_PACK, B.PDKV_OP_UNPACK, B.PDKV_OP_TRANSFER)}
+
     def synchronize(self, stream: Optional[int] = None) -> None:
         """Wait for the session's stream (and raise if a kernel reported an error)."""
         self.status(stream)

@@ -449,3 +449,64 @@ def test_plan_in_caller_workspace(oracle):
         B.pdkv_plan_destroy(plan)
         dst_t.copy_(dev(sent)); torch.cuda.synchronize()
     B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
+
+
+def test_pinned_and_autotuned_launch_shapes(oracle):
+    """Per-plan launch shapes (set by hand, or found by pdkv_plan_autotune) change how
+    the work is spread over threads, never the bytes; shapes found for a geometry
+    are handed to later plans of that geometry unless "autotune_reuse" is off."""
+    from paper_2408_08147_b200.session import TransferSession
+
+    lens = np.array([700, 33, 1500, 16, 260], np.int32)
+    w = W.build_workload("rows-of-160-bytes", 11, num_layers=2, num_kv_heads=8, head_dim=80, elem_bytes=2,
+                         seq_len=lens, src_layout=W.BLOCK_MAJOR, src_block=16, dst_layout=W.LAYER_MAJOR,
+                         dst_block=128, src_slack=1.2, dst_slack=1.2)
+    G = w.dst.block_tokens
+    src = W.fill_pool_numpy(w.src, w.seed)
+    sent = W.sentinel_pool_numpy(w.dst)
+    want_dst = sent.copy()
+    oracle.transfer(w.src, src, w.dst, want_dst, w.batch)
+    want_buf = np.zeros(oracle.buffer_elems(w.batch, G, w.src), np.uint16)
+    oracle.pack(w.src, src, w.batch, G, want_buf)
+    src_t, dst_t = dev(src), dev(sent)
+    torch.cuda.synchronize()
+    ops = (B.PDKV_OP_PACK, B.PDKV_OP_UNPACK, B.PDKV_OP_TRANSFER)
+    try:
+        with TransferSession(w.src, src_t, w.dst, dst_t, w.batch) as s:
+            buf_t = torch.zeros(s.buffer_bytes, dtype=torch.uint8, device="cuda")
+            for shape in [(640, 1, 2), (160, 4, 3), (96, 2, 8), (1024, 1, 1), (256, 8, 1)]:
+                for op in ops:
+                    B.pdkv_plan_set_shape(s.plan, op, *shape)
+                buf_t.zero_()
+                dst_t.copy_(dev(sent))
+                torch.cuda.synchronize()
+                s.pack(buf_t); s.unpack(buf_t); s.status()
+                assert np.array_equal(host(buf_t), want_buf), f"pack with shape {shape}"
+                assert np.array_equal(host(dst_t), want_dst), f"unpack with shape {shape}"
+                dst_t.copy_(dev(sent))
+                torch.cuda.synchronize()
+                s.transfer(); s.status()
+                assert np.array_equal(host(dst_t), want_dst), f"transfer with shape {shape}"
+            for op in ops:
+                B.pdkv_plan_set_shape(s.plan, op, 0, 0, 0)
+            buf_t.zero_()
+            dst_t.copy_(dev(sent))
+            torch.cuda.synchronize()
+            found = s.autotune(buf_t)
+            s.status()
+            for op, (threads, unroll, ctas) in found.items():
+                assert (threads, unroll, ctas) == (0, 0, 0) or (threads % 32 == 0 and unroll in (1, 2, 4) and ctas >= 1)
+            # autotuning runs the real operations: buffer and decode pool hold the batch afterwards
+            assert np.array_equal(host(buf_t), want_buf)
+            assert np.array_equal(host(dst_t), want_dst)
+            dst_t.copy_(dev(sent))
+            torch.cuda.synchronize()
+            s.transfer(); s.status()
+            assert np.array_equal(host(dst_t), want_dst), f"transfer with the shapes found: {found}"
+            with TransferSession(w.src, src_t, w.dst, dst_t, w.batch) as again:      # same geometry: shapes handed on
+                assert {op: B.pdkv_plan_shape(again.plan, op) for op in ops} == found
+            B.pdkv_tune("autotune_reuse", 0)
+            with TransferSession(w.src, src_t, w.dst, dst_t, w.batch) as fresh:
+                assert all(B.pdkv_plan_shape(fresh.plan, op) == (0, 0, 0) for op in ops)
+    finally:
+        B.pdkv_tune("autotune_reuse", 1)

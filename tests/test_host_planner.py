@@ -354,3 +354,28 @@ def test_tile_offsets_in_petabyte_pools_need_64_bits():
     assert got == want and max(a for a, _, _ in got) > 2 ** 49
     B.pdkv_plan_destroy(plan)
     B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
+
+
+def test_launch_shapes_of_a_plan():
+    w = W.make_config(3, num_layers=2, n_req=3, max_len=300)
+    ps, pd = _pools(w)
+    plan = _plan(w, ps, pd)
+    try:
+        for op in (B.PDKV_OP_PACK, B.PDKV_OP_UNPACK, B.PDKV_OP_TRANSFER):
+            assert B.pdkv_plan_shape(plan, op) == (0, 0, 0)          # built-in choice
+        B.pdkv_plan_set_shape(plan, B.PDKV_OP_TRANSFER, 384, 2, 3)
+        assert B.pdkv_plan_shape(plan, B.PDKV_OP_TRANSFER) == (384, 2, 3)
+        assert B.pdkv_plan_shape(plan, B.PDKV_OP_PACK) == (0, 0, 0)
+        for bad in [(100, 1, 2), (2048, 1, 2), (256, 3, 2), (256, 4, 0), (0, 4, 2)]:
+            with pytest.raises(B.PdkvError) as e:
+                B.pdkv_plan_set_shape(plan, B.PDKV_OP_PACK, *bad)
+            assert e.value.status == B.PDKV_ERR_INVALID_ARG
+        B.pdkv_plan_set_shape(plan, B.PDKV_OP_TRANSFER, 0, 0, 0)
+        assert B.pdkv_plan_shape(plan, B.PDKV_OP_TRANSFER) == (0, 0, 0)
+        with pytest.raises(B.PdkvError) as e:                         # a host-only plan cannot be timed
+            B.pdkv_plan_autotune(plan)
+        assert e.value.status == B.PDKV_ERR_INVALID_ARG
+    finally:
+        B.pdkv_plan_destroy(plan)
+        B.pdkv_pool_destroy(ps)
+        B.pdkv_pool_destroy(pd)
