@@ -167,8 +167,9 @@ int pdkv_plan_destroy(pdkv_plan *plan);
  * in exactly one or two passes.  About ten candidate shapes are launched a few
  * times each over some or all layers of the batch, for pack and unpack (only
  * if `buf` is given: device, at least pdkv_plan_buffer() bytes) and for
- * transfer; a shape replaces the built-in one only if it is more than 1.5%
- * faster.  The operations are the real ones: afterwards `buf` holds the packed
+ * transfer; a shape replaces the built-in one only if it is more than 2.5%
+ * faster.  With a block-major pool the strip skew (see "lc_skew") is also timed
+ * the other way round than its stride rule decides, and kept on the same terms.  The operations are the real ones: afterwards `buf` holds the packed
  * layers and the decode pool the transferred layers that were used for timing
  * (with an unpack-only plan `buf` must already hold a packed batch).  The
  * call synchronises `stream` repeatedly; it is meant for set-up time, once per
@@ -176,11 +177,12 @@ int pdkv_plan_destroy(pdkv_plan *plan);
  * remembered for every later plan of the process with the same pool
  * geometries and tile sizes.  Explicit "threads" / "unroll" tunables override
  * it.  Plans with small tiles (under 8 KiB) are left alone.  (No counterpart in
- * the paper.)  pdkv_plan_shape() reports what a plan uses (zeros: built-in).
+ * the paper.)  pdkv_plan_shape() reports what a plan uses (zeros: built-in;
+ * lc_skew -1: by the stride rule, 0: none, > 0: that many strips).
  * Errors: INVALID_ARG, BUFFER_TOO_SMALL, CUDA. */
 int pdkv_plan_autotune(pdkv_plan *plan, void *buf, size_t buf_bytes, void *stream);
 int pdkv_plan_shape(const pdkv_plan *plan, int op, int32_t *threads, int32_t *unroll,
-                    int32_t *ctas_per_sm);
+                    int32_t *ctas_per_sm, int32_t *lc_skew);
 /* Pin the launch shape of one operation of this plan by hand (threads: multiple of
  * 32 up to 1024, clamped to what the register budget allows; unroll: 1, 2, 4 or 8;
  * ctas_per_sm: 1..32); all three zero returns to the built-in choice.  Not

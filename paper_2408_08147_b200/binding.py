@@ -210,10 +210,12 @@ def pdkv_plan_autotune(plan: int, buf_ptr: int = 0, buf_bytes: int = 0, stream: 
 
 
 def pdkv_plan_shape(plan: int, op: int):
-    """(threads, unroll, ctas_per_sm) the plan uses for ``op``; zeros = the built-in choice."""
-    t, u, c = C.c_int32(), C.c_int32(), C.c_int32()
-    _check(lib().pdkv_plan_shape(C.c_void_p(plan), op, C.byref(t), C.byref(u), C.byref(c)), "pdkv_plan_shape")
-    return int(t.value), int(u.value), int(c.value)
+    """(threads, unroll, ctas_per_sm, lc_skew) the plan uses for ``op``; zeros = the built-in
+    shape, lc_skew -1 = by the stride rule."""
+    t, u, c, k = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32()
+    _check(lib().pdkv_plan_shape(C.c_void_p(plan), op, C.byref(t), C.byref(u), C.byref(c), C.byref(k)),
+           "pdkv_plan_shape")
+    return int(t.value), int(u.value), int(c.value), int(k.value)
 
 
 def pdkv_plan_set_shape(plan: int, op: int, threads: int, unroll: int, ctas_per_sm: int) -> None:

@@ -87,6 +87,7 @@ struct pdkv_plan {
     // launch shape found by pdkv_plan_autotune() for each operation; threads == 0: not tuned
     struct Shape {
         int threads = 0, unroll = 0, ctas_per_sm = 0;
+        int skew = -1;   // strip skew: -1 by the stride rule, 0 none, > 0 this many strips
     } shape[3];
 };
 
@@ -273,18 +274,25 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
         if (skew < 0) {
             skew = 0;
             shift = 0;
+            bool have_pool = false;
             auto consider = [&](const pdkv_pool &pool) {
-                if (skew || pool.d.layout != PDKV_LAYOUT_BLOCK_MAJOR) return;
+                if (have_pool || pool.d.layout != PDKV_LAYOUT_BLOCK_MAJOR) return;
                 const uint64_t strip = (uint64_t)pool.d.block_tokens * (uint64_t)pl->hrow_bytes;
                 uint64_t odd = 2ull * (uint64_t)pl->L * strip;
                 while (odd && !(odd & 1ull)) odd >>= 1;
-                if (odd % 3 && odd % 5 && odd % 17) return;
+                const bool slow_stride = !(odd % 3 && odd % 5 && odd % 17);
+                if (!slow_stride && pl->shape[op].skew <= 0) return;
+                have_pool = true;
                 skew = 16;
                 const uint64_t per_block = pl->max_tile_bytes > 0 ? strip / (uint64_t)pl->max_tile_bytes : 1;
                 while ((2ull << shift) <= per_block) ++shift;
             };
             if (op != PDKV_OP_UNPACK && pl->has_src) consider(pl->src);   // the pool that is read comes first
             if (op != PDKV_OP_PACK && pl->has_dst) consider(pl->dst);
+            // pdkv_plan_autotune() may have measured that this batch is better off without the rule's
+            // skew (0), or with one although the rule sees no reason (> 0; needs a block-major pool)
+            if (pl->shape[op].skew == 0) skew = 0;
+            else if (pl->shape[op].skew > 0 && have_pool) skew = pl->shape[op].skew;
         }
         while (skew > 1 && skew > p.n_lc) skew >>= 1;   // a power of two within the strips of this call
         p.lc_skew = p.lc_fastest ? 0 : (int32_t)skew;
@@ -696,9 +704,9 @@ int pdkv_plan_autotune(pdkv_plan *plan, void *buf, size_t buf_bytes, void *strea
         if (e0) cudaEventDestroy(e0);
         return cuda_fail(e, "cudaEventCreate");
     }
-    // enough layers for a launch of a few hundred MiB, all of them for small batches
+    // enough layers for a launch of a few GiB (fewer strips change how a sweep behaves), all of them for small batches
     int layers = plan->L;
-    const uint64_t want_bytes = 1ull << 30;
+    const uint64_t want_bytes = 4ull << 30;
     if (plan->payload_bytes > want_bytes)
         layers = (int)std::max<uint64_t>(2, std::min<uint64_t>((uint64_t)plan->L, (uint64_t)plan->L * want_bytes / plan->payload_bytes));
     layers = std::min(layers, (int)plan->L);
@@ -754,12 +762,31 @@ int pdkv_plan_autotune(pdkv_plan *plan, void *buf, size_t buf_bytes, void *strea
             plan->shape[op] = cand[i];
             float ms = 0.f;
             rc = time_ms(op, &ms);
-            if (rc == PDKV_OK && ms < 0.985f * best_ms) {   // a candidate must win by more than the noise
+            if (rc == PDKV_OK && ms < 0.975f * best_ms) {   // a candidate must win by more than the noise (2.5%)
                 best_ms = ms;
                 best = cand[i];
             }
         }
         plan->shape[op] = best;
+        // the strip skew the other way round: on where the stride rule leaves it off, off where it is on
+        if (rc == PDKV_OK && pdkv::tunables().lc_skew < 0 && pdkv::tunables().lc_fastest == 0) {
+            const pdkv_pool *pools[2] = {op != PDKV_OP_UNPACK && plan->has_src ? &plan->src : nullptr,
+                                         op != PDKV_OP_PACK && plan->has_dst ? &plan->dst : nullptr};
+            bool block_major = false, rule_on = false;
+            for (const pdkv_pool *pool : pools) {
+                if (!pool || pool->d.layout != PDKV_LAYOUT_BLOCK_MAJOR) continue;
+                block_major = true;
+                uint64_t odd = 2ull * (uint64_t)plan->L * (uint64_t)pool->d.block_tokens * (uint64_t)plan->hrow_bytes;
+                while (odd && !(odd & 1ull)) odd >>= 1;
+                rule_on = rule_on || !(odd % 3 && odd % 5 && odd % 17);
+            }
+            if (block_major && 2 * layers >= 16) {
+                plan->shape[op].skew = rule_on ? 0 : 16;
+                float ms = 0.f;
+                rc = time_ms(op, &ms);
+                if (!(rc == PDKV_OK && ms < 0.975f * best_ms)) plan->shape[op].skew = -1;
+            }
+        }
     }
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
@@ -782,6 +809,7 @@ int pdkv_plan_set_shape(pdkv_plan *plan, int op, int32_t threads, int32_t unroll
         plan->shape[op] = pdkv_plan::Shape();
         return PDKV_OK;
     }
+    plan->shape[op].skew = -1;
     if (threads < 32 || threads > 1024 || threads % 32 || (unroll != 1 && unroll != 2 && unroll != 4 && unroll != 8) ||
         ctas_per_sm < 1 || ctas_per_sm > 32)
         return PDKV_ERR_INVALID_ARG;
@@ -791,9 +819,11 @@ int pdkv_plan_set_shape(pdkv_plan *plan, int op, int32_t threads, int32_t unroll
     return PDKV_OK;
 }
 
-int pdkv_plan_shape(const pdkv_plan *plan, int op, int32_t *threads, int32_t *unroll, int32_t *ctas_per_sm)
+int pdkv_plan_shape(const pdkv_plan *plan, int op, int32_t *threads, int32_t *unroll, int32_t *ctas_per_sm,
+                    int32_t *lc_skew)
 {
     if (!plan || op < 0 || op > 2) return PDKV_ERR_INVALID_ARG;
+    if (lc_skew) *lc_skew = plan->shape[op].skew;
     if (threads) *threads = plan->shape[op].threads;
     if (unroll) *unroll = plan->shape[op].unroll;
     if (ctas_per_sm) *ctas_per_sm = plan->shape[op].ctas_per_sm;

@@ -494,8 +494,9 @@ def test_pinned_and_autotuned_launch_shapes(oracle):
             torch.cuda.synchronize()
             found = s.autotune(buf_t)
             s.status()
-            for op, (threads, unroll, ctas) in found.items():
+            for op, (threads, unroll, ctas, skew) in found.items():
                 assert (threads, unroll, ctas) == (0, 0, 0) or (threads % 32 == 0 and unroll in (1, 2, 4) and ctas >= 1)
+                assert skew in (-1, 0, 16)
             # autotuning runs the real operations: buffer and decode pool hold the batch afterwards
             assert np.array_equal(host(buf_t), want_buf)
             assert np.array_equal(host(dst_t), want_dst)
@@ -507,6 +508,6 @@ def test_pinned_and_autotuned_launch_shapes(oracle):
                 assert {op: B.pdkv_plan_shape(again.plan, op) for op in ops} == found
             B.pdkv_tune("autotune_reuse", 0)
             with TransferSession(w.src, src_t, w.dst, dst_t, w.batch) as fresh:
-                assert all(B.pdkv_plan_shape(fresh.plan, op) == (0, 0, 0) for op in ops)
+                assert all(B.pdkv_plan_shape(fresh.plan, op) == (0, 0, 0, -1) for op in ops)
     finally:
         B.pdkv_tune("autotune_reuse", 1)

@@ -362,16 +362,16 @@ def test_launch_shapes_of_a_plan():
     plan = _plan(w, ps, pd)
     try:
         for op in (B.PDKV_OP_PACK, B.PDKV_OP_UNPACK, B.PDKV_OP_TRANSFER):
-            assert B.pdkv_plan_shape(plan, op) == (0, 0, 0)          # built-in choice
+            assert B.pdkv_plan_shape(plan, op) == (0, 0, 0, -1)      # built-in choice, skew by the stride rule
         B.pdkv_plan_set_shape(plan, B.PDKV_OP_TRANSFER, 384, 2, 3)
-        assert B.pdkv_plan_shape(plan, B.PDKV_OP_TRANSFER) == (384, 2, 3)
-        assert B.pdkv_plan_shape(plan, B.PDKV_OP_PACK) == (0, 0, 0)
+        assert B.pdkv_plan_shape(plan, B.PDKV_OP_TRANSFER) == (384, 2, 3, -1)
+        assert B.pdkv_plan_shape(plan, B.PDKV_OP_PACK) == (0, 0, 0, -1)
         for bad in [(100, 1, 2), (2048, 1, 2), (256, 3, 2), (256, 4, 0), (0, 4, 2)]:
             with pytest.raises(B.PdkvError) as e:
                 B.pdkv_plan_set_shape(plan, B.PDKV_OP_PACK, *bad)
             assert e.value.status == B.PDKV_ERR_INVALID_ARG
         B.pdkv_plan_set_shape(plan, B.PDKV_OP_TRANSFER, 0, 0, 0)
-        assert B.pdkv_plan_shape(plan, B.PDKV_OP_TRANSFER) == (0, 0, 0)
+        assert B.pdkv_plan_shape(plan, B.PDKV_OP_TRANSFER) == (0, 0, 0, -1)
         with pytest.raises(B.PdkvError) as e:                         # a host-only plan cannot be timed
             B.pdkv_plan_autotune(plan)
         assert e.value.status == B.PDKV_ERR_INVALID_ARG
