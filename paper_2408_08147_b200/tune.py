@@ -7,6 +7,9 @@ re-run it and pin the winners with ``pdkv_tune``::
     python -m paper_2408_08147_b200.tune --config 3 --kv-heads 2
     python -m paper_2408_08147_b200.tune --config 4 --ops fused --grid wide
 
+(``pdkv_plan_autotune`` does a short version of this inside the library, per
+plan, for the launch shape alone.)
+
 Timing is bench-like: the selected operations are issued back to back on one
 stream and each one's CUDA-event time is averaged over ``--reps`` rounds.
 """
@@ -46,6 +49,8 @@ def main(argv=None) -> int:
     ap.add_argument("--n-req", type=int, default=0)
     ap.add_argument("--kv-heads", type=int, default=0)
     ap.add_argument("--elem-bytes", type=int, default=0)
+    ap.add_argument("--head-dim", type=int, default=0)
+    ap.add_argument("--num-layers", type=int, default=0)
     ap.add_argument("--ops", default="pack,unpack,fused")
     ap.add_argument("--grid", default="quick", choices=sorted(GRIDS))
     ap.add_argument("--reps", type=int, default=5)
@@ -57,7 +62,7 @@ def main(argv=None) -> int:
 
     kw = {}
     for key, val in (("src_block", a.src_block), ("n_req", a.n_req), ("num_kv_heads", a.kv_heads),
-                     ("elem_bytes", a.elem_bytes)):
+                     ("elem_bytes", a.elem_bytes), ("head_dim", a.head_dim), ("num_layers", a.num_layers)):
         if val:
             kw[key] = val
     if a.layouts:
