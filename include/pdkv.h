@@ -164,8 +164,8 @@ int pdkv_plan_destroy(pdkv_plan *plan);
  * choice is tuned for Llama-shaped geometries (32 KiB tiles of 256-byte rows);
  * other head sizes, head counts or block sizes can run several percent -- for
  * 160-byte rows up to 30% -- faster with a shape that covers one of their tiles
- * in exactly one or two passes.  About ten candidate shapes are launched a few
- * times each over some or all layers of the batch, for pack and unpack (only
+ * in exactly one or two passes.  About ten candidate shapes are launched four
+ * times each over all layers of the batch, for pack and unpack (only
  * if `buf` is given: device, at least pdkv_plan_buffer() bytes) and for
  * transfer; a shape replaces the built-in one only if it is more than 2.5%
  * faster.  With a block-major pool the strip skew (see "lc_skew") is also timed

@@ -329,10 +329,18 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
             cfg.unroll = tuned.unroll;
             cfg.ctas_per_sm = tuned.ctas_per_sm;
         }
+        // Tiles of more than half but less than a full 256 x 4 pass (head sizes, head counts or
+        // block sizes that are not powers of two): that one pass, whatever the class of copy.
+        const int64_t max_vecs = pl->max_tile_bytes / cfg.vec_bytes;
+        const bool odd_tile = !use_tuned && cfg.unroll == 0 && cfg.threads == 0 && max_vecs > 512 && max_vecs < 1024;
+        if (odd_tile) {
+            cfg.unroll = 4;
+            cfg.threads = 256;
+        }
         if (cfg.unroll == 0) cfg.unroll = (flat || small) ? 1 : 4;
         if (cfg.threads == 0) cfg.threads = (flat || small) ? 512 : 256;
         cfg.group_threads = (int)pdkv::tunables().group_threads;
-        if (use_tuned && cfg.group_threads == 0) cfg.group_threads = cfg.threads;
+        if ((use_tuned || odd_tile) && cfg.group_threads == 0) cfg.group_threads = cfg.threads;
         if (cfg.group_threads == 0) {
             const int64_t vecs = std::max<int64_t>(1, pl->mean_tile_bytes[op] / cfg.vec_bytes);
             const int64_t want = vecs / ((flat || small) ? 2 : cfg.unroll);
@@ -704,12 +712,8 @@ int pdkv_plan_autotune(pdkv_plan *plan, void *buf, size_t buf_bytes, void *strea
         if (e0) cudaEventDestroy(e0);
         return cuda_fail(e, "cudaEventCreate");
     }
-    // enough layers for a launch of a few GiB (fewer strips change how a sweep behaves), all of them for small batches
-    int layers = plan->L;
-    const uint64_t want_bytes = 4ull << 30;
-    if (plan->payload_bytes > want_bytes)
-        layers = (int)std::max<uint64_t>(2, std::min<uint64_t>((uint64_t)plan->L, (uint64_t)plan->L * want_bytes / plan->payload_bytes));
-    layers = std::min(layers, (int)plan->L);
+    // whole-model launches: a subset of the layers has fewer strips per sweep and was seen to rank shapes differently
+    const int layers = plan->L;
 
     int rc = PDKV_OK;
     auto run = [&](int op) -> int {
