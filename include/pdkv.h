@@ -25,6 +25,12 @@
  *     host<->device copy, no synchronisation; after one call outside capture
  *     they can be recorded into a CUDA graph (e.g. the per-layer sequence of a
  *     model) and replayed.
+ *   - A plan is immutable once created and may be used from any thread: it
+ *     carries its own copy of the launch tunables (pdkv_tune) as they stood at
+ *     creation, so a later pdkv_tune() -- from this or another thread -- changes
+ *     only plans created afterwards.  (pdkv_plan_autotune / pdkv_plan_set_shape
+ *     are the two calls that modify a plan; they are set-up calls and must not
+ *     run beside launches of the same plan.)
  *   - Elements are opaque: `elem_bytes` bytes are moved bit for bit (NaN
  *     payloads and -0 survive).
  *
@@ -34,9 +40,9 @@
  *   PDKV_LAYOUT_LAYER_MAJOR  [layer][K/V][block][head][token][dim]
  *       elem = ((((l*2 + c)*NB + b)*H + h)*B + tt)*D + d
  *
- * Contiguous buffer (Sec. 3.5: K and V of each layer "one after another";
- * a layer's offset and length follow from prompt length, hidden size and
- * precision): requests are concatenated in batch order without padding; inside
+ * Contiguous buffer (Sec. 3.5: the K and V tensors of consecutive layers lie
+ * back to back; a layer's offset and length follow from prompt length, hidden
+ * size and precision): requests are concatenated in batch order without padding; inside
  * request r the order is [layer][K/V][kept token][head][dim].  With n_r kept
  * tokens, layer l of request r is the byte range
  *       [ off_r + l*2*n_r*H*D*E ,  + 2*n_r*H*D*E ),
@@ -245,13 +251,22 @@ int pdkv_transfer(const pdkv_plan *plan, int layer_begin, int layer_end, void *s
  *     per block boundary); beyond that PDKV_ERR_LIMIT is returned and nothing
  *     is enqueued.  Raise "tile_bytes" or split the batch.
  *   - The first call on each device looks up the device address of the scratch
- *     array (with that device current).  Make that first call outside any
- *     stream capture.
+ *     array (with that device current) and loads the library's device image;
+ *     make it once at start-up, before HBM is handed to the engine's allocator.
+ *   - The call stages the tile list from host memory that it frees on return,
+ *     so it cannot be recorded: when `stream` is capturing it returns
+ *     INVALID_ARG and enqueues nothing.  Graph users need plans
+ *     (pdkv_plan_create_in places one in caller-owned memory).
+ *   - Launch shape, work order and strip skew come from the same chooser as
+ *     pdkv_transfer() with the tunables as they stand at the call; "variant"
+ *     and "debug_bounds" are not honoured (register-copy kernel, no checks).
  *   - Every call on a device reuses the same scratch, which still holds the
  *     previous call's tiles; the call rewrites what it needs (including the
  *     words that must start at zero) on `stream` before its kernel runs.  Two
  *     calls whose GPU work can overlap (different streams without an ordering
- *     between them) race on it: order them, or use plans.
+ *     between them) race on it, and so do two host threads that enqueue on the
+ *     same stream at the same time (their clear / copy / kernel steps may
+ *     interleave): order them, or use plans.
  *   - The tile list is copied from pageable host memory, so the call may block
  *     until earlier work on `stream` has finished.
  * Errors: INVALID_ARG, GEOMETRY, TABLE, LIMIT, CUDA, NOMEM. */
@@ -261,8 +276,8 @@ int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
                           const pdkv_batch_desc *batch, int layer_begin, int layer_end,
                           void *stream);
 
-/* Baseline: the block-by-block transfer of Sec. 2.3 ("transfer one by one"),
- * one copy or one kernel launch per prefill block issued from a host loop.
+/* Baseline: the block-by-block transfer that Sec. 2.3 describes as the natural
+ * consequence of block-fixed pools, one copy or one kernel launch per prefill block issued from a host loop.
  * Same result as pdkv_transfer over all layers. */
 int pdkv_transfer_blockwise(const pdkv_plan *plan, void *stream);
 
@@ -295,8 +310,14 @@ int pdkv_plan_block_bytes(const pdkv_plan *plan, uint64_t *src_bytes, uint64_t *
  *                       transfer over all layers on the slot's stream --
  *                       preceded by pdkv_upload_blocks() if `host_src_pool` is
  *                       given and followed by pdkv_download_blocks() if
- *                       `host_dst_pool` is given (either may be NULL).  Returns a
- *                       ticket.  If every slot is taken it returns PDKV_ERR_BUSY at
+ *                       `host_dst_pool` is given (either may be NULL).  A slot's
+ *                       stream is ordered after nothing the caller has enqueued:
+ *                       pass in `wait_event` (a cudaEvent_t as void*, or NULL) an
+ *                       event recorded after the work that produces the prefill
+ *                       blocks and after the last reader of the decode blocks
+ *                       about to be overwritten -- the slot waits for it on the
+ *                       device -- or synchronise with that work on the host
+ *                       before the call.  Returns a ticket.  If every slot is taken it returns PDKV_ERR_BUSY at
  *                       once and enqueues nothing: nothing waits inside the library,
  *                       the caller retries when a request completes.
  *   pdkv_queue_poll     *done = 1 once the slot's transfer has finished (its
@@ -312,7 +333,7 @@ int pdkv_plan_block_bytes(const pdkv_plan *plan, uint64_t *src_bytes, uint64_t *
 int pdkv_queue_create(const pdkv_pool *src, const pdkv_pool *dst, int device, int capacity,
                       pdkv_queue **out);
 int pdkv_queue_submit(pdkv_queue *queue, const pdkv_batch_desc *batch, const void *host_src_pool,
-                      void *host_dst_pool, int64_t *ticket);
+                      void *host_dst_pool, void *wait_event, int64_t *ticket);
 int pdkv_queue_poll(pdkv_queue *queue, int64_t ticket, int *done);
 int pdkv_queue_wait(pdkv_queue *queue, int64_t ticket);
 int pdkv_queue_release(pdkv_queue *queue, int64_t ticket);
@@ -345,7 +366,22 @@ int pdkv_plan_tiles(const pdkv_plan *plan, int op, const pdkv_tile **tiles, int6
  * kernel returned early) or PDKV_ERR_CUDA. */
 int pdkv_plan_status(const pdkv_plan *plan, void *stream);
 
-/* Process-wide tunables, read when a plan is created or a call is launched:
+/* What a plan will launch for `op` over layers [layer_begin, layer_end): the
+ * result of the library's chooser (class of copy, tile sizes, stride rule,
+ * autotuned or pinned shape) applied to the tunables frozen in the plan.  Works
+ * on host-only ("dry_run") plans too.  pdkv_plan_option() reads one frozen
+ * tunable by its pdkv_tune() key.  Errors: INVALID_ARG. */
+typedef struct {
+    int32_t threads, unroll, ctas_per_sm, group_threads, vec_bytes, max_ctas;
+    int32_t lc_skew, lc_skew_shift, lc_fastest, chunked, src_order, variant, debug_bounds;
+} pdkv_launch_shape;
+int pdkv_plan_launch_shape(const pdkv_plan *plan, int op, int layer_begin, int layer_end,
+                           pdkv_launch_shape *out);
+int pdkv_plan_option(const pdkv_plan *plan, const char *key, int64_t *value);
+
+/* Process-wide tunables: the defaults of plans created afterwards.  pdkv_plan_create()
+ * copies them into the plan (pdkv_transfer_noalloc() reads them at the call); changing
+ * them never affects a plan that already exists.
  *   "tile_bytes"     target bytes moved per tile (default 32768)
  *   "ctas_per_sm"    persistent CTAs per SM (default 2)
  *   "max_ctas"       cap on the grid size, 0 = none (default).  A small grid
@@ -380,6 +416,12 @@ int pdkv_plan_status(const pdkv_plan *plan, void *stream);
  *                    block together); chosen automatically with "lc_skew" -1
  *   "chunked"        1: each CTA takes one contiguous run of work items instead
  *                    of every gridDim-th one (default 0)
+ *   "src_order"      order in which the threads of a CTA walk the rows of a tile whose
+ *                    two sides differ in order (one token-major, one head-major): 0 in
+ *                    the order of the side written, 1 of the side read, -1 (default)
+ *                    automatic: read order when a row (D*E bytes) is not a multiple of
+ *                    64 bytes -- a lone read of such a row fetches a sector more than it
+ *                    uses -- else write order
  *   "debug_bounds"   1: kernels range-check every access and skip bad ones
  *   "debug_shrink"   with "debug_bounds": pretend each side is N bytes shorter, so
  *                    that the refusal path can be exercised on valid memory

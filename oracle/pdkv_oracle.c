@@ -48,11 +48,6 @@ typedef struct {
     const uint8_t *skip;         /* parallel to dst_tbl, or NULL */
 } okv_batch;
 
-int64_t okv_pool_elems(const okv_geom *g)
-{
-    return (int64_t)g->NB * g->L * 2 * g->B * g->H * g->D;
-}
-
 static int64_t pool_off(const okv_geom *g, int64_t b, int64_t l, int64_t c,
                         int64_t tt, int64_t h, int64_t d)
 {

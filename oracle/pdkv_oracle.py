@@ -47,8 +47,6 @@ def _load():
     global _lib
     if _lib is None:
         lib = C.CDLL(build())
-        lib.okv_pool_elems.restype = C.c_int64
-        lib.okv_pool_elems.argtypes = [C.POINTER(_Geom)]
         lib.okv_kept_tokens.restype = C.c_int64
         lib.okv_kept_tokens.argtypes = [C.POINTER(_Batch), C.c_int]
         lib.okv_request_offset.restype = C.c_int64

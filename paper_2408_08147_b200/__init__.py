@@ -4,9 +4,9 @@
 ``session``   convenience holder of the C handles of one batch
 ``workloads`` seeded synthetic inputs (no transfer arithmetic)
 ``build``     builds the shared library with nvcc
-``tune``      ``python -m paper_2408_08147_b200.tune``: sweep the launch tunables on a workload
+``p2d``       sender rank / receiver rank protocol over ``torch.distributed``
 
 Nothing here falls back to a CPU path: without the built library every call
 raises.
 """
-__all__ = ["binding", "session", "workloads", "build", "tune"]
+__all__ = ["binding", "session", "workloads", "build", "p2d"]

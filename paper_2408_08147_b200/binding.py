@@ -43,7 +43,7 @@ EXPORTS = (
     "pdkv_plan_status", "pdkv_upload_blocks", "pdkv_download_blocks", "pdkv_plan_block_bytes",
     "pdkv_queue_create", "pdkv_queue_submit", "pdkv_queue_poll", "pdkv_queue_wait", "pdkv_queue_release",
     "pdkv_queue_stats", "pdkv_queue_destroy", "pdkv_tune", "pdkv_tune_get", "pdkv_strerror",
-    "pdkv_plan_autotune", "pdkv_plan_shape", "pdkv_plan_set_shape",
+    "pdkv_plan_autotune", "pdkv_plan_shape", "pdkv_plan_set_shape", "pdkv_plan_launch_shape", "pdkv_plan_option",
 )
 
 
@@ -62,6 +62,12 @@ class pdkv_batch_desc(C.Structure):
 class pdkv_tile(C.Structure):
     _fields_ = [("src_off", C.c_int64), ("dst_off", C.c_int64), ("ntok", C.c_int32),
                 ("n_kept", C.c_int32)]
+
+
+class pdkv_launch_shape(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in ("threads", "unroll", "ctas_per_sm", "group_threads", "vec_bytes", "max_ctas",
+                                         "lc_skew", "lc_skew_shift", "lc_fastest", "chunked", "src_order", "variant",
+                                         "debug_bounds")]
 
 
 TILE_DTYPE = np.dtype([("src_off", "<i8"), ("dst_off", "<i8"), ("ntok", "<i4"), ("n_kept", "<i4")])
@@ -109,7 +115,9 @@ def lib() -> C.CDLL:
     L.pdkv_download_blocks.argtypes = [vp, vp, vp]
     L.pdkv_plan_block_bytes.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     L.pdkv_queue_create.argtypes = [vp, vp, C.c_int, C.c_int, C.POINTER(vp)]
-    L.pdkv_queue_submit.argtypes = [vp, C.POINTER(pdkv_batch_desc), vp, vp, C.POINTER(i64)]
+    L.pdkv_queue_submit.argtypes = [vp, C.POINTER(pdkv_batch_desc), vp, vp, vp, C.POINTER(i64)]
+    L.pdkv_plan_launch_shape.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.POINTER(pdkv_launch_shape)]
+    L.pdkv_plan_option.argtypes = [vp, C.c_char_p, C.POINTER(i64)]
     L.pdkv_queue_poll.argtypes = [vp, i64, C.POINTER(C.c_int)]
     L.pdkv_queue_wait.argtypes = [vp, i64]
     L.pdkv_queue_release.argtypes = [vp, i64]
@@ -216,6 +224,21 @@ def pdkv_plan_shape(plan: int, op: int):
     _check(lib().pdkv_plan_shape(C.c_void_p(plan), op, C.byref(t), C.byref(u), C.byref(c), C.byref(k)),
            "pdkv_plan_shape")
     return int(t.value), int(u.value), int(c.value), int(k.value)
+
+
+def pdkv_plan_launch_shape(plan: int, op: int, layer_begin: int, layer_end: int) -> dict:
+    """What the plan launches for ``op`` over the layer range, as a dict of the fields of
+    ``pdkv_launch_shape``."""
+    out = pdkv_launch_shape()
+    _check(lib().pdkv_plan_launch_shape(C.c_void_p(plan), op, layer_begin, layer_end, C.byref(out)),
+           "pdkv_plan_launch_shape")
+    return {k: int(getattr(out, k)) for k, _ in pdkv_launch_shape._fields_}
+
+
+def pdkv_plan_option(plan: int, key: str) -> int:
+    v = C.c_int64()
+    _check(lib().pdkv_plan_option(C.c_void_p(plan), key.encode(), C.byref(v)), f"pdkv_plan_option({key})")
+    return int(v.value)
 
 
 def pdkv_plan_set_shape(plan: int, op: int, threads: int, unroll: int, ctas_per_sm: int) -> None:
@@ -326,12 +349,14 @@ def pdkv_queue_create(src_pool: int, dst_pool: int, device: int, capacity: int) 
 
 
 def pdkv_queue_submit(queue: int, seq_len, src_tbl_off, src_tbl, dst_tbl_off, dst_tbl, dst_skip=None,
-                      host_src_ptr: Optional[int] = None, host_dst_ptr: Optional[int] = None):
-    """Returns a ticket, or ``None`` when every receive slot is taken."""
+                      host_src_ptr: Optional[int] = None, host_dst_ptr: Optional[int] = None,
+                      wait_event: Optional[int] = None):
+    """Returns a ticket, or ``None`` when every receive slot is taken.  ``wait_event`` is a
+    ``cudaEvent_t`` handle (e.g. ``torch.cuda.Event.cuda_event``) the slot's stream waits for."""
     b = _BatchArrays(seq_len, src_tbl_off, src_tbl, dst_tbl_off, dst_tbl, dst_skip)
     t = C.c_int64()
     rc = lib().pdkv_queue_submit(C.c_void_p(queue), C.byref(b.desc), C.c_void_p(host_src_ptr),
-                                 C.c_void_p(host_dst_ptr), C.byref(t))
+                                 C.c_void_p(host_dst_ptr), C.c_void_p(wait_event), C.byref(t))
     if rc == PDKV_ERR_BUSY:
         return None
     _check(rc, "pdkv_queue_submit")

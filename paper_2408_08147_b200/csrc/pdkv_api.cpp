@@ -32,6 +32,7 @@ struct BlockGroup {     // one prefill block's share of the fused transfer (base
 
 thread_local std::string g_cuda_msg;
 thread_local bool g_host_only_plan = false;  // set only around pdkv::create_host_plan()
+thread_local unsigned g_plan_ops = 7u;       // tile lists to build (bit per pdkv_op); narrowed only there
 
 int cuda_fail(cudaError_t e, const char *what)
 {
@@ -84,6 +85,7 @@ struct pdkv_plan {
     int64_t max_tile_bytes = 0;
     int64_t mean_tile_bytes[3] = {0, 0, 0};   // per operation, over its tile list
     int sm_count = 1;
+    pdkv::LaunchOptions opt;   // the tunables as they stood when the plan was created
     // launch shape found by pdkv_plan_autotune() for each operation; threads == 0: not tuned
     struct Shape {
         int threads = 0, unroll = 0, ctas_per_sm = 0;
@@ -249,9 +251,9 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     pdkv::CopyParams p;
     p.src = src;
     p.dst = dst;
-    if (pdkv::tunables().debug_bounds && pdkv::tunables().debug_shrink > 0) {
-        p.src.size = std::max<int64_t>(0, p.src.size - pdkv::tunables().debug_shrink);
-        p.dst.size = std::max<int64_t>(0, p.dst.size - pdkv::tunables().debug_shrink);
+    if (pl->opt.debug_bounds && pl->opt.debug_shrink > 0) {
+        p.src.size = std::max<int64_t>(0, p.src.size - pl->opt.debug_shrink);
+        p.dst.size = std::max<int64_t>(0, p.dst.size - pl->opt.debug_shrink);
     }
     p.tiles = pl->dev_tiles[op];
     p.tile_begin = tile_begin;
@@ -260,103 +262,21 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     p.n_lc = 2 * (l1 - l0);
     p.H = pl->H;
     p.row_bytes = (int32_t)pl->row_bytes;
-    p.lc_fastest = (int32_t)pdkv::tunables().lc_fastest;
-    p.chunked = (int32_t)pdkv::tunables().chunked;
-    {   // Strip skew (see pdkv_tune "lc_skew").  Automatic: only for calls that read (or, failing
-        // that, write) a block-major pool whose block stride, stripped of its factors of two, is
-        // divisible by 3, 5 or 17 (e.g. 80 layers x 64 tokens x 2 KiB = 5 x 4 MiB).  With such
-        // strides the same-offset strips of many blocks, which one sweep touches at the same
-        // time, collide in DRAM (measured on 37 strides: reads 4-12% and writes 2% slower, every
-        // odd part sharing a factor with 255 and no other); skewing the strip by the block's
-        // position in the batch spreads them and recovers most of it.  Tiles of one block keep
-        // the same skew so that its strip is still moved in one piece.
-        int64_t skew = pdkv::tunables().lc_skew, shift = pdkv::tunables().lc_skew_shift;
-        if (skew < 0) {
-            skew = 0;
-            shift = 0;
-            bool have_pool = false;
-            auto consider = [&](const pdkv_pool &pool) {
-                if (have_pool || pool.d.layout != PDKV_LAYOUT_BLOCK_MAJOR) return;
-                const uint64_t strip = (uint64_t)pool.d.block_tokens * (uint64_t)pl->hrow_bytes;
-                uint64_t odd = 2ull * (uint64_t)pl->L * strip;
-                while (odd && !(odd & 1ull)) odd >>= 1;
-                const bool slow_stride = !(odd % 3 && odd % 5 && odd % 17);
-                if (!slow_stride && pl->shape[op].skew <= 0) return;
-                have_pool = true;
-                skew = 16;
-                const uint64_t per_block = pl->max_tile_bytes > 0 ? strip / (uint64_t)pl->max_tile_bytes : 1;
-                while ((2ull << shift) <= per_block) ++shift;
-            };
-            if (op != PDKV_OP_UNPACK && pl->has_src) consider(pl->src);   // the pool that is read comes first
-            if (op != PDKV_OP_PACK && pl->has_dst) consider(pl->dst);
-            // pdkv_plan_autotune() may have measured that this batch is better off without the rule's
-            // skew (0), or with one although the rule sees no reason (> 0; needs a block-major pool)
-            if (pl->shape[op].skew == 0) skew = 0;
-            else if (pl->shape[op].skew > 0 && have_pool) skew = pl->shape[op].skew;
-        }
-        while (skew > 1 && skew > p.n_lc) skew >>= 1;   // a power of two within the strips of this call
-        p.lc_skew = p.lc_fastest ? 0 : (int32_t)skew;
-        p.lc_skew_shift = (int32_t)shift;
-    }
+    pdkv::ResolvedLaunch r;
+    pdkv::resolve_launch(pl, op, src, dst, p.n_lc, pl->sm_count, &r);
+    p.lc_fastest = r.lc_fastest;
+    p.chunked = r.chunked;
+    p.lc_skew = r.lc_skew;
+    p.lc_skew_shift = r.lc_skew_shift;
+    p.src_order = r.src_order;
+    p.group_threads = 0;
     p.status = pl->dev_status;
-    pdkv::LaunchConfig cfg;
-    cfg.vec_bytes = pl->vec_bytes;
-    if (pl->vec_bytes == 16 && pdkv::tunables().vec32 && pl->row_bytes % 32 == 0 &&
-        ((reinterpret_cast<uintptr_t>(src.base) | reinterpret_cast<uintptr_t>(dst.base)) & 31u) == 0)
-        cfg.vec_bytes = 32;
-    cfg.unroll = (int)pdkv::tunables().unroll;
-    cfg.threads = (int)pdkv::tunables().threads;
-    cfg.ctas_per_sm = (int)pdkv::tunables().ctas_per_sm;
-    cfg.max_ctas = (int)pdkv::tunables().max_ctas;
-    cfg.sm_count = pl->sm_count;
-    cfg.variant = (int)pdkv::tunables().variant;
-    cfg.elem_bytes = pl->E;
-    cfg.check_bounds = pdkv::tunables().debug_bounds != 0;
-    {   // Automatic launch shape, measured best per class of copy on B200.  Full tiles
-        // (about 32 KiB): a flat copy (token-major on both sides) runs 512 threads with
-        // one access in flight each, i.e. two passes per tile; a copy with a head-major
-        // side runs 256 threads with four, i.e. one pass per tile.  Batches of small
-        // tiles (few KV heads, short blocks): groups of threads that cover a tile in two
-        // passes of one access each, 32 threads at least.
-        const int64_t hrow = pl->hrow_bytes, row = pl->row_bytes;
-        const bool flat = src.head_stride == row && src.tok_stride == hrow && dst.head_stride == row &&
-                          dst.tok_stride == hrow;
-        const bool small = pl->mean_tile_bytes[op] < 24 * 1024;
-        const pdkv_plan::Shape &tuned = pl->shape[op];
-        const bool use_tuned = tuned.threads > 0 && cfg.unroll == 0 && cfg.threads == 0;
-        if (use_tuned) {   // found by pdkv_plan_autotune(): the whole CTA works on one tile
-            cfg.threads = tuned.threads;
-            cfg.unroll = tuned.unroll;
-            cfg.ctas_per_sm = tuned.ctas_per_sm;
-        }
-        // Tiles of more than half but less than a full 256 x 4 pass (head sizes, head counts or
-        // block sizes that are not powers of two): that one pass, whatever the class of copy.
-        const int64_t max_vecs = pl->max_tile_bytes / cfg.vec_bytes;
-        const bool odd_tile = !use_tuned && cfg.unroll == 0 && cfg.threads == 0 && max_vecs > 512 && max_vecs < 1024;
-        if (odd_tile) {
-            cfg.unroll = 4;
-            cfg.threads = 256;
-        }
-        if (cfg.unroll == 0) cfg.unroll = (flat || small) ? 1 : 4;
-        if (cfg.threads == 0) cfg.threads = (flat || small) ? 512 : 256;
-        cfg.group_threads = (int)pdkv::tunables().group_threads;
-        if ((use_tuned || odd_tile) && cfg.group_threads == 0) cfg.group_threads = cfg.threads;
-        if (cfg.group_threads == 0) {
-            const int64_t vecs = std::max<int64_t>(1, pl->mean_tile_bytes[op] / cfg.vec_bytes);
-            const int64_t want = vecs / ((flat || small) ? 2 : cfg.unroll);
-            int g = 32;
-            while (g < want && g < cfg.threads) g *= 2;
-            cfg.group_threads = g;
-        }
-    }
-    cfg.stages = (int)pdkv::tunables().stages;
-    cfg.max_tile_bytes = pl->max_tile_bytes;
     cudaError_t e;
-    if (cfg.variant >= 1 && pdkv::bulk_supported(cfg, p.row_bytes)) {
-        cfg.vec_bytes = 16;
-        e = pdkv::launch_bulk(p, cfg, stream);
+    if (r.cfg.variant >= 1 && pdkv::bulk_supported(r.cfg, p.row_bytes)) {
+        r.cfg.vec_bytes = 16;
+        e = pdkv::launch_bulk(p, r.cfg, stream);
     } else {
-        e = pdkv::launch_copy(p, cfg, stream);
+        e = pdkv::launch_copy(p, r.cfg, stream);
     }
     if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
     return PDKV_OK;
@@ -410,13 +330,38 @@ Tunables &tunables()
 
 namespace pdkv {
 
-int create_host_plan(const pdkv_pool *src, const pdkv_pool *dst, const pdkv_batch_desc *batch,
+int create_host_plan(const pdkv_pool *src, const pdkv_pool *dst, const pdkv_batch_desc *batch, unsigned op_mask,
                      pdkv_plan **out)
 {
     g_host_only_plan = true;
+    g_plan_ops = op_mask & 7u;
     const int rc = pdkv_plan_create(src, dst, 0, batch, nullptr, out);
+    g_plan_ops = 7u;
     g_host_only_plan = false;
     return rc;
+}
+
+LaunchOptions snapshot_options()
+{
+    const Tunables &t = tunables();
+    LaunchOptions o;
+    o.ctas_per_sm = (int)t.ctas_per_sm;
+    o.max_ctas = (int)t.max_ctas;
+    o.threads = (int)t.threads;
+    o.unroll = (int)t.unroll;
+    o.vec32 = (int)t.vec32;
+    o.lc_fastest = (int)t.lc_fastest;
+    o.group_threads = (int)t.group_threads;
+    o.chunked = (int)t.chunked;
+    o.lc_skew = (int)t.lc_skew;
+    o.lc_skew_shift = (int)t.lc_skew_shift;
+    o.debug_bounds = (int)t.debug_bounds;
+    o.debug_shrink = t.debug_shrink;
+    o.variant = (int)t.variant;
+    o.stages = (int)t.stages;
+    o.src_order = (int)t.src_order;
+    o.tile_bytes = t.tile_bytes;
+    return o;
 }
 
 void describe_transfer(const pdkv_plan *plan, Side *src, Side *dst, int *H, int *row_bytes,
@@ -429,6 +374,105 @@ void describe_transfer(const pdkv_plan *plan, Side *src, Side *dst, int *H, int 
     *vec_bytes = plan->vec_bytes;
     *num_layers = plan->L;
     *device = plan->device;
+}
+
+void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &dst, int n_lc, int sm_count,
+                    ResolvedLaunch *out)
+{
+    const LaunchOptions &o = pl->opt;
+    out->lc_fastest = o.lc_fastest;
+    out->chunked = o.chunked;
+    {   // Strip skew (see pdkv_tune "lc_skew").  Automatic: only for calls that read (or, failing
+        // that, write) a block-major pool whose block stride, stripped of its factors of two, is
+        // divisible by 3, 5 or 17 (e.g. 80 layers x 64 tokens x 2 KiB = 5 x 4 MiB).  With such
+        // strides the same-offset strips of many blocks, which one sweep touches at the same
+        // time, collide in DRAM (measured on 37 strides: reads 4-12% and writes 2% slower, every
+        // odd part sharing a factor with 255 and no other); skewing the strip by the block's
+        // position in the batch spreads them and recovers most of it.  Tiles of one block keep
+        // the same skew so that its strip is still moved in one piece.
+        int64_t skew = o.lc_skew, shift = o.lc_skew_shift;
+        if (skew < 0) {
+            skew = 0;
+            shift = 0;
+            bool have_pool = false;
+            auto consider = [&](const pdkv_pool &pool) {
+                if (have_pool || pool.d.layout != PDKV_LAYOUT_BLOCK_MAJOR) return;
+                const uint64_t strip = (uint64_t)pool.d.block_tokens * (uint64_t)pl->hrow_bytes;
+                uint64_t odd = 2ull * (uint64_t)pl->L * strip;
+                while (odd && !(odd & 1ull)) odd >>= 1;
+                const bool slow_stride = !(odd % 3 && odd % 5 && odd % 17);
+                if (!slow_stride && pl->shape[op].skew <= 0) return;
+                have_pool = true;
+                skew = 16;
+                const uint64_t per_block = pl->max_tile_bytes > 0 ? strip / (uint64_t)pl->max_tile_bytes : 1;
+                while ((2ull << shift) <= per_block) ++shift;
+            };
+            if (op != PDKV_OP_UNPACK && pl->has_src) consider(pl->src);   // the pool that is read comes first
+            if (op != PDKV_OP_PACK && pl->has_dst) consider(pl->dst);
+            // pdkv_plan_autotune() may have measured that this batch is better off without the rule's
+            // skew (0), or with one although the rule sees no reason (> 0; needs a block-major pool)
+            if (pl->shape[op].skew == 0) skew = 0;
+            else if (pl->shape[op].skew > 0 && have_pool) skew = pl->shape[op].skew;
+        }
+        while (skew > 1 && skew > n_lc) skew >>= 1;   // a power of two within the strips of this call
+        out->lc_skew = out->lc_fastest ? 0 : (int32_t)skew;
+        out->lc_skew_shift = (int32_t)shift;
+    }
+    LaunchConfig &cfg = out->cfg;
+    cfg.vec_bytes = pl->vec_bytes;
+    if (pl->vec_bytes == 16 && o.vec32 && pl->row_bytes % 32 == 0 &&
+        ((reinterpret_cast<uintptr_t>(src.base) | reinterpret_cast<uintptr_t>(dst.base)) & 31u) == 0)
+        cfg.vec_bytes = 32;
+    cfg.unroll = o.unroll;
+    cfg.threads = o.threads;
+    cfg.ctas_per_sm = o.ctas_per_sm;
+    cfg.max_ctas = o.max_ctas;
+    cfg.sm_count = sm_count;
+    cfg.variant = o.variant;
+    cfg.elem_bytes = pl->E;
+    cfg.check_bounds = o.debug_bounds != 0;
+    const int64_t hrow = pl->hrow_bytes, row = pl->row_bytes;
+    const bool flat = src.head_stride == row && src.tok_stride == hrow && dst.head_stride == row &&
+                      dst.tok_stride == hrow;
+    {   // Automatic launch shape, measured best per class of copy on B200.  Full tiles
+        // (about 32 KiB): a flat copy (token-major on both sides) runs 512 threads with
+        // one access in flight each, i.e. two passes per tile; a copy with a head-major
+        // side runs 256 threads with four, i.e. one pass per tile.  Batches of small
+        // tiles (few KV heads, short blocks): groups of threads that cover a tile in two
+        // passes of one access each, 32 threads at least.
+        const bool small = pl->mean_tile_bytes[op] < 24 * 1024;
+        const pdkv_plan::Shape &tuned = pl->shape[op];
+        const bool use_tuned = tuned.threads > 0 && cfg.unroll == 0 && cfg.threads == 0;
+        if (use_tuned) {   // found by pdkv_plan_autotune(): the whole CTA works on one tile
+            cfg.threads = tuned.threads;
+            cfg.unroll = tuned.unroll;
+            cfg.ctas_per_sm = tuned.ctas_per_sm;
+        }
+        // Tiles of more than half but less than a full 256 x 4 pass (head sizes, head counts or
+        // block sizes that are not powers of two): that one pass, whatever the class of copy.
+        const int64_t max_vecs = pl->max_tile_bytes / cfg.vec_bytes;
+        const bool odd_tile = !use_tuned && cfg.unroll == 0 && cfg.threads == 0 && max_vecs > 512 && max_vecs < 1024;
+        if (odd_tile) {
+            cfg.unroll = 4;
+            cfg.threads = 256;
+        }
+        if (cfg.unroll == 0) cfg.unroll = (flat || small) ? 1 : 4;
+        if (cfg.threads == 0) cfg.threads = (flat || small) ? 512 : 256;
+        cfg.group_threads = o.group_threads;
+        if ((use_tuned || odd_tile) && cfg.group_threads == 0) cfg.group_threads = cfg.threads;
+        if (cfg.group_threads == 0) {
+            const int64_t vecs = std::max<int64_t>(1, pl->mean_tile_bytes[op] / cfg.vec_bytes);
+            const int64_t want = vecs / ((flat || small) ? 2 : cfg.unroll);
+            int g = 32;
+            while (g < want && g < cfg.threads) g *= 2;
+            cfg.group_threads = g;
+        }
+    }
+    // Row order inside a tile (see CopyParams::src_order): rows that are not whole 64-byte
+    // pairs of sectors are walked in the order of the side that is read.
+    out->src_order = o.src_order >= 0 ? o.src_order : ((!flat && row % 64 != 0) ? 1 : 0);
+    cfg.stages = o.stages;
+    cfg.max_tile_bytes = pl->max_tile_bytes;
 }
 
 int report_cuda_error(cudaError_t e, const char *what) { return cuda_fail(e, what); }
@@ -522,6 +566,7 @@ int pdkv_plan_create_in(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip
         pl->row_bytes = (int64_t)pl->D * pl->E;
         pl->hrow_bytes = pl->row_bytes * pl->H;
         pl->n_req = batch->n_req;
+        pl->opt = pdkv::snapshot_options();
 
         int rc;
         if (src && (rc = check_table(batch->src_tbl_off, batch->src_tbl, batch->n_req, batch->seq_len,
@@ -613,7 +658,7 @@ int pdkv_plan_create_in(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip
         // Tile size cap.  The kernels split a vector index with multiply-high
         // divisions that are exact while dividend * divisor < 2^32, so the cap
         // also keeps vectors * vectors-per-row and rows * max(H, tokens) below it.
-        int64_t cap_tok = std::max<int64_t>(1, pdkv::tunables().tile_bytes / pl->hrow_bytes);
+        int64_t cap_tok = std::max<int64_t>(1, pl->opt.tile_bytes / pl->hrow_bytes);
         {
             const int64_t vpr = pl->row_bytes / pl->vec_bytes;
             const int64_t max_b = std::max<int64_t>(src ? src->d.block_tokens : 1, dst ? dst->d.block_tokens : 1);
@@ -625,9 +670,9 @@ int pdkv_plan_create_in(const pdkv_pool *src, const pdkv_pool *dst, int32_t skip
             while (cap_tok > 1 && !exact(cap_tok)) cap_tok /= 2;
             if (!exact(cap_tok)) return PDKV_ERR_GEOMETRY;
         }
-        if (src) build_tiles(*pl, PDKV_OP_PACK, *batch, cap_tok);
-        if (dst) build_tiles(*pl, PDKV_OP_UNPACK, *batch, cap_tok);
-        if (src && dst) build_tiles(*pl, PDKV_OP_TRANSFER, *batch, cap_tok);
+        if (src && (g_plan_ops & 1u)) build_tiles(*pl, PDKV_OP_PACK, *batch, cap_tok);
+        if (dst && (g_plan_ops & 2u)) build_tiles(*pl, PDKV_OP_UNPACK, *batch, cap_tok);
+        if (src && dst && (g_plan_ops & 4u)) build_tiles(*pl, PDKV_OP_TRANSFER, *batch, cap_tok);
         for (int op = 0; op < 3; ++op) {
             if (pl->tiles[op].size() > (size_t)INT32_MAX) return PDKV_ERR_INVALID_ARG;
             int64_t sum = 0;
@@ -773,7 +818,7 @@ int pdkv_plan_autotune(pdkv_plan *plan, void *buf, size_t buf_bytes, void *strea
         }
         plan->shape[op] = best;
         // the strip skew the other way round: on where the stride rule leaves it off, off where it is on
-        if (rc == PDKV_OK && pdkv::tunables().lc_skew < 0 && pdkv::tunables().lc_fastest == 0) {
+        if (rc == PDKV_OK && plan->opt.lc_skew < 0 && plan->opt.lc_fastest == 0) {
             const pdkv_pool *pools[2] = {op != PDKV_OP_UNPACK && plan->has_src ? &plan->src : nullptr,
                                          op != PDKV_OP_PACK && plan->has_dst ? &plan->dst : nullptr};
             bool block_major = false, rule_on = false;
@@ -831,6 +876,58 @@ int pdkv_plan_shape(const pdkv_plan *plan, int op, int32_t *threads, int32_t *un
     if (threads) *threads = plan->shape[op].threads;
     if (unroll) *unroll = plan->shape[op].unroll;
     if (ctas_per_sm) *ctas_per_sm = plan->shape[op].ctas_per_sm;
+    return PDKV_OK;
+}
+
+int pdkv_plan_option(const pdkv_plan *plan, const char *key, int64_t *value)
+{
+    if (!plan || !key || !value) return PDKV_ERR_INVALID_ARG;
+    const pdkv::LaunchOptions &o = plan->opt;
+    const std::string k(key);
+    if (k == "tile_bytes") *value = o.tile_bytes;
+    else if (k == "ctas_per_sm") *value = o.ctas_per_sm;
+    else if (k == "max_ctas") *value = o.max_ctas;
+    else if (k == "threads") *value = o.threads;
+    else if (k == "unroll") *value = o.unroll;
+    else if (k == "vec32") *value = o.vec32;
+    else if (k == "lc_fastest") *value = o.lc_fastest;
+    else if (k == "chunked") *value = o.chunked;
+    else if (k == "lc_skew") *value = o.lc_skew;
+    else if (k == "lc_skew_shift") *value = o.lc_skew_shift;
+    else if (k == "group_threads") *value = o.group_threads;
+    else if (k == "debug_bounds") *value = o.debug_bounds;
+    else if (k == "debug_shrink") *value = o.debug_shrink;
+    else if (k == "variant") *value = o.variant;
+    else if (k == "stages") *value = o.stages;
+    else if (k == "src_order") *value = o.src_order;
+    else return PDKV_ERR_INVALID_ARG;
+    return PDKV_OK;
+}
+
+int pdkv_plan_launch_shape(const pdkv_plan *plan, int op, int layer_begin, int layer_end, pdkv_launch_shape *out)
+{
+    if (!plan || !out || op < 0 || op > 2 || !layers_ok(plan, layer_begin, layer_end)) return PDKV_ERR_INVALID_ARG;
+    if ((op != PDKV_OP_UNPACK && !plan->has_src) || (op != PDKV_OP_PACK && !plan->has_dst))
+        return PDKV_ERR_INVALID_ARG;
+    // the buffer's base is taken as 32-byte aligned, as device allocations are
+    const pdkv::Side buf = buffer_side(nullptr, 0, plan->row_bytes, plan->hrow_bytes);
+    const pdkv::Side s = op == PDKV_OP_UNPACK ? buf : pool_side(plan->src, plan->row_bytes, plan->hrow_bytes);
+    const pdkv::Side d = op == PDKV_OP_PACK ? buf : pool_side(plan->dst, plan->row_bytes, plan->hrow_bytes);
+    pdkv::ResolvedLaunch r;
+    pdkv::resolve_launch(plan, op, s, d, 2 * (layer_end - layer_begin), plan->sm_count, &r);
+    out->threads = r.cfg.threads;
+    out->unroll = r.cfg.unroll;
+    out->ctas_per_sm = r.cfg.ctas_per_sm;
+    out->group_threads = r.cfg.group_threads;
+    out->vec_bytes = r.cfg.vec_bytes;
+    out->max_ctas = r.cfg.max_ctas;
+    out->lc_skew = r.lc_skew;
+    out->lc_skew_shift = r.lc_skew_shift;
+    out->lc_fastest = r.lc_fastest;
+    out->chunked = r.chunked;
+    out->src_order = r.src_order;
+    out->variant = r.cfg.variant;
+    out->debug_bounds = r.cfg.check_bounds ? 1 : 0;
     return PDKV_OK;
 }
 
@@ -1061,6 +1158,7 @@ int pdkv_tune(const char *key, int64_t value)
     else if (k == "stages" && value >= 2 && value <= 16) t.stages = value;
     else if (k == "dry_run" && (value == 0 || value == 1)) t.dry_run = value;
     else if (k == "autotune_reuse" && (value == 0 || value == 1)) t.autotune_reuse = value;
+    else if (k == "src_order" && value >= -1 && value <= 1) t.src_order = value;
     else return PDKV_ERR_INVALID_ARG;
     return PDKV_OK;
 }
@@ -1087,6 +1185,7 @@ int pdkv_tune_get(const char *key, int64_t *value)
     else if (k == "stages") *value = t.stages;
     else if (k == "dry_run") *value = t.dry_run;
     else if (k == "autotune_reuse") *value = t.autotune_reuse;
+    else if (k == "src_order") *value = t.src_order;
     else return PDKV_ERR_INVALID_ARG;
     return PDKV_OK;
 }

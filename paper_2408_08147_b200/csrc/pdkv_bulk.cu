@@ -3,8 +3,8 @@
 // of shared-memory stages, one tile per stage.  No data passes through
 // registers, so the kernel occupies one warp and a few registers per CTA: this
 // is the "operator" form of RecvScatter that leaves the SMs' issue slots and
-// register file to whatever else runs in the stream (Sec. 3.5, "does not
-// interrupt the computation of other operators").
+// register file to whatever else runs in the stream (Sec. 3.5: as an operator the
+// scatter runs beside the stream's other operators without holding them up).
 //
 // A tile is staged in *destination order*.  Towards a head-major pool that is
 // [head][token][row]: the H stores are contiguous runs of ntok*ROW bytes and

@@ -102,7 +102,11 @@ copy_tiles_kernel(const CopyParams p)
     const uint32_t vpr = (uint32_t)p.row_bytes / W;  // vectors per row
     const uint32_t H = (uint32_t)p.H;
     const int64_t hrow = (int64_t)p.H * p.row_bytes;
-    const bool head_inner = p.dst.tok_stride >= p.dst.head_stride;
+    // Rows of a tile are walked in the order of the side that is written, or (src_order) of the
+    // side that is read.  When a row is not a whole number of 64-byte sector pairs (160-byte
+    // rows of 80 bf16, say) a lone row read drags in the neighbouring row's half pair; walking
+    // in the order of the reads makes those neighbours part of the same pass.
+    const bool head_inner = p.src_order ? p.src.tok_stride >= p.src.head_stride : p.dst.tok_stride >= p.dst.head_stride;
     const bool flat = p.src.head_stride == p.row_bytes && p.src.tok_stride == hrow &&
                       p.dst.head_stride == p.row_bytes && p.dst.tok_stride == hrow;
     const int64_t n_work = (int64_t)p.n_tiles * p.n_lc;

@@ -43,6 +43,7 @@ struct CopyParams {
     int32_t lc_skew;       // power of two <= n_lc, or <= 1 for none: tile t works on strip (s + ((t >> shift) & (skew-1))) mod n_lc in sweep s
     int32_t lc_skew_shift;
     int32_t group_threads;  // threads that cooperate on one work item (set by the launcher)
+    int32_t src_order;      // 1: the rows of a tile are walked in the order of the side that is read, 0: of the side written
     unsigned long long *status;  // [0] != 0: an access was refused; [1] offending offset
 };
 
@@ -108,13 +109,36 @@ struct Tunables {
     std::atomic<int64_t> stages{3};
     std::atomic<int64_t> dry_run{0};
     std::atomic<int64_t> autotune_reuse{1};
+    std::atomic<int64_t> src_order{-1};   // -1: by the row size (see CopyParams::src_order)
 };
 Tunables &tunables();
 
-// Used by the no-allocation entry point (its own translation unit).
+// The tunables that steer a launch, copied into a plan when it is created: a plan keeps
+// launching the way it was set up, whatever pdkv_tune() is told afterwards (by this or
+// another thread).  pdkv_tune() only sets the defaults of plans created later.
+struct LaunchOptions {
+    int ctas_per_sm = 2, max_ctas = 0, threads = 0, unroll = 0, vec32 = 1, lc_fastest = 0, group_threads = 0,
+        chunked = 0, lc_skew = -1, lc_skew_shift = 0, debug_bounds = 0, variant = 0, stages = 3, src_order = -1;
+    int64_t debug_shrink = 0;
+    int64_t tile_bytes = 32768;
+};
+LaunchOptions snapshot_options();
+
+// Everything launch_copy()/launch_bulk() need besides the sides, the tile list and the layer range.
+struct ResolvedLaunch {
+    LaunchConfig cfg;
+    int32_t lc_fastest, chunked, lc_skew, lc_skew_shift, src_order;
+};
+
+// Used by the no-allocation entry point and the retrieval queue (their own translation units).
 // A host-only plan: validated batch and tile lists, no CUDA call, nothing on the device.
-int create_host_plan(const pdkv_pool *src, const pdkv_pool *dst, const pdkv_batch_desc *batch,
+// `op_mask` (bit per pdkv_op) says which tile lists to build.
+int create_host_plan(const pdkv_pool *src, const pdkv_pool *dst, const pdkv_batch_desc *batch, unsigned op_mask,
                      pdkv_plan **out);
+// The launch shape, work order and strip skew the plan uses for `op` between these two sides over
+// `n_lc` (layer, K/V) strips: the one chooser behind every entry point.
+void resolve_launch(const pdkv_plan *plan, int op, const Side &src, const Side &dst, int n_lc, int sm_count,
+                    ResolvedLaunch *out);
 void describe_transfer(const pdkv_plan *plan, Side *src, Side *dst, int *H, int *row_bytes,
                        int *vec_bytes, int *num_layers, int *device);
 int report_cuda_error(cudaError_t e, const char *what);

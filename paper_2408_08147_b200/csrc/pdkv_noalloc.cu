@@ -59,8 +59,16 @@ extern "C" int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
                                      void *stream)
 {
     if (!src || !dst || !batch) return PDKV_ERR_INVALID_ARG;
-    PlanHolder plan;  // host memory only: validated batch and its tile lists
-    int rc = pdkv::create_host_plan(src, dst, batch, &plan.p);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    {   // The tile list below is staged from host memory that this call frees on return, so the
+        // call cannot be recorded: a capturing stream is refused before anything is enqueued.
+        cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+        cudaError_t ce = cudaStreamIsCapturing(st, &capturing);
+        if (ce != cudaSuccess) return pdkv::report_cuda_error(ce, "cudaStreamIsCapturing");
+        if (capturing != cudaStreamCaptureStatusNone) return PDKV_ERR_INVALID_ARG;
+    }
+    PlanHolder plan;  // host memory only: validated batch and the tile list of the fused transfer
+    int rc = pdkv::create_host_plan(src, dst, batch, 1u << PDKV_OP_TRANSFER, &plan.p);
     if (rc != PDKV_OK) return rc;
 
     pdkv::CopyParams p;
@@ -84,7 +92,6 @@ extern "C" int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
 
     rc = PDKV_OK;
     DeviceSlot slot;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((e = device_slot(device, &slot)) != cudaSuccess) {
         rc = pdkv::report_cuda_error(e, "cudaGetSymbolAddress");
     } else if ((e = cudaMemsetAsync(slot.scratch, 0, kHeaderBytes, st)) != cudaSuccess) {
@@ -93,7 +100,6 @@ extern "C" int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
                                     cudaMemcpyHostToDevice, st)) != cudaSuccess) {
         rc = pdkv::report_cuda_error(e, "cudaMemcpyAsync");
     } else {
-        const pdkv::Tunables &t = pdkv::tunables();
         p.tiles = reinterpret_cast<const pdkv::Tile *>(slot.scratch + kHeaderBytes);
         p.tile_begin = 0;
         p.n_tiles = (int32_t)n_tiles;
@@ -101,28 +107,19 @@ extern "C" int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
         p.n_lc = 2 * (layer_end - layer_begin);
         p.H = H;
         p.row_bytes = row_bytes;
-        p.lc_fastest = (int32_t)t.lc_fastest;
-        p.chunked = (int32_t)t.chunked;
-        p.lc_skew = 0;
-        p.lc_skew_shift = 0;
+        // launch shape, work order and strip skew from the chooser every plan-based call uses
+        pdkv::ResolvedLaunch r;
+        pdkv::resolve_launch(plan.p, PDKV_OP_TRANSFER, p.src, p.dst, p.n_lc, slot.sm_count, &r);
+        p.lc_fastest = r.lc_fastest;
+        p.chunked = r.chunked;
+        p.lc_skew = r.lc_skew;
+        p.lc_skew_shift = r.lc_skew_shift;
+        p.src_order = r.src_order;
+        p.group_threads = 0;
         p.status = reinterpret_cast<unsigned long long *>(slot.scratch);
-        pdkv::LaunchConfig cfg;
-        cfg.vec_bytes = vec_bytes;
-        if (vec_bytes == 16 && t.vec32 && row_bytes % 32 == 0 &&
-            ((reinterpret_cast<uintptr_t>(p.src.base) | reinterpret_cast<uintptr_t>(p.dst.base)) & 31u) == 0)
-            cfg.vec_bytes = 32;
-        cfg.unroll = t.unroll ? (int)t.unroll : 4;
-        cfg.threads = t.threads ? (int)t.threads : 256;
-        cfg.ctas_per_sm = (int)t.ctas_per_sm;
-        cfg.max_ctas = (int)t.max_ctas;
-        cfg.sm_count = slot.sm_count;
-        cfg.variant = 0;
-        cfg.elem_bytes = 0;
-        cfg.group_threads = cfg.threads;
-        cfg.stages = 0;
-        cfg.max_tile_bytes = 0;
-        cfg.check_bounds = false;
-        if ((e = pdkv::launch_copy(p, cfg, st)) != cudaSuccess) rc = pdkv::report_cuda_error(e, "kernel launch");
+        r.cfg.variant = 0;            // the register-copy kernel: it needs nothing but the tile list
+        r.cfg.check_bounds = false;   // there is no plan to report a refusal through
+        if ((e = pdkv::launch_copy(p, r.cfg, st)) != cudaSuccess) rc = pdkv::report_cuda_error(e, "kernel launch");
     }
     if (prev != device) cudaSetDevice(prev);
     return rc;

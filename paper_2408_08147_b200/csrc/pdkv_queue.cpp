@@ -80,7 +80,7 @@ int pdkv_queue_create(const pdkv_pool *src, const pdkv_pool *dst, int device, in
 }
 
 int pdkv_queue_submit(pdkv_queue *q, const pdkv_batch_desc *batch, const void *host_src_pool,
-                      void *host_dst_pool, int64_t *ticket)
+                      void *host_dst_pool, void *wait_event, int64_t *ticket)
 {
     if (ticket) *ticket = -1;
     if (!q || !batch || !ticket) return PDKV_ERR_INVALID_ARG;
@@ -97,7 +97,7 @@ int pdkv_queue_submit(pdkv_queue *q, const pdkv_batch_desc *batch, const void *h
     }
     int rc;
     if (q->host_only) {
-        rc = pdkv::create_host_plan(q->src, q->dst, batch, &slot->plan);
+        rc = pdkv::create_host_plan(q->src, q->dst, batch, 7u, &slot->plan);
         if (rc != PDKV_OK) return rc;
     } else {
         DevGuard guard(q->device);
@@ -107,7 +107,11 @@ int pdkv_queue_submit(pdkv_queue *q, const pdkv_batch_desc *batch, const void *h
         if (rc == PDKV_ERR_BUFFER_TOO_SMALL)   // a batch with more tiles than the slot's workspace holds
             rc = pdkv_plan_create(q->src, q->dst, 0, batch, slot->stream, &slot->plan);
         if (rc != PDKV_OK) return rc;
-        if (host_src_pool) rc = pdkv_upload_blocks(slot->plan, host_src_pool, slot->stream);
+        if (wait_event) {   // the slot's stream runs beside the caller's: order it after the producer of the blocks
+            cudaError_t e = cudaStreamWaitEvent(slot->stream, static_cast<cudaEvent_t>(wait_event), 0);
+            if (e != cudaSuccess) rc = pdkv::report_cuda_error(e, "cudaStreamWaitEvent");
+        }
+        if (rc == PDKV_OK && host_src_pool) rc = pdkv_upload_blocks(slot->plan, host_src_pool, slot->stream);
         if (rc == PDKV_OK) rc = pdkv_transfer(slot->plan, 0, pdkv::plan_num_layers(slot->plan), slot->stream);
         if (rc == PDKV_OK && host_dst_pool) rc = pdkv_download_blocks(slot->plan, host_dst_pool, slot->stream);
         if (rc == PDKV_OK) {

@@ -88,8 +88,9 @@ def test_step_bytes_accounting_matches_the_library():
             b = w.batch
             plan = B.pdkv_plan_create(ps, pd, 0, b.seq_len, b.src_tbl_off, b.src_tbl, b.dst_tbl_off,
                                       b.dst_tbl, b.dst_skip)
-            total = sum(sum(B.pdkv_plan_traffic(plan, op)) for op in range(3))
-            assert total == bench.step_bytes_of(w)
+            per_op = [sum(B.pdkv_plan_traffic(plan, op)) for op in range(3)]
+            assert sum(per_op) == bench.step_bytes_of(w)
+            assert per_op == [bench.op_bytes_of(w)[k] for k in ("pack", "unpack", "fused")]
             B.pdkv_plan_destroy(plan)
             B.pdkv_pool_destroy(ps)
             B.pdkv_pool_destroy(pd)

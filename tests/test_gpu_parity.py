@@ -408,7 +408,7 @@ def test_sender_only_and_receiver_only_plans(oracle, idx, kw):
         L = w.src.num_layers
         for l in range(L):                                  # per-layer trigger: offset and length per layer
             sender.pack(send_buf, (l, l + 1))
-        recv_buf.copy_(send_buf)                            # "transfer all the data as a whole"
+        recv_buf.copy_(send_buf)                            # the whole buffer in one copy (Sec. 3.5)
         receiver.unpack(recv_buf)
         torch.cuda.synchronize()
         assert np.array_equal(host(dst_t), want)

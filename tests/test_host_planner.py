@@ -379,3 +379,71 @@ def test_launch_shapes_of_a_plan():
         B.pdkv_plan_destroy(plan)
         B.pdkv_pool_destroy(ps)
         B.pdkv_pool_destroy(pd)
+
+
+def test_plans_keep_the_tunables_they_were_created_with():
+    """A plan copies the launch tunables when it is created: two plans made under different
+    settings keep launching differently after the settings are put back, and a later
+    pdkv_tune() changes neither."""
+    w = W.make_config(3, num_layers=4, n_req=6, max_len=900)
+    ps, pd = _pools(w)
+    names = ("threads", "unroll", "ctas_per_sm", "lc_skew", "max_ctas", "debug_bounds", "src_order")
+    before = {k: B.pdkv_tune_get(k) for k in names}
+    try:
+        default_plan = _plan(w, ps, pd)
+        for k, v in dict(threads=128, unroll=2, ctas_per_sm=5, lc_skew=8, max_ctas=64, debug_bounds=1,
+                         src_order=1).items():
+            B.pdkv_tune(k, v)
+        tuned_plan = _plan(w, ps, pd)
+    finally:
+        for k, v in before.items():
+            B.pdkv_tune(k, v)
+    L = w.src.num_layers
+    a = B.pdkv_plan_launch_shape(default_plan, B.PDKV_OP_TRANSFER, 0, L)
+    b = B.pdkv_plan_launch_shape(tuned_plan, B.PDKV_OP_TRANSFER, 0, L)
+    # block-major 16-token blocks -> layer-major: a row-permuting copy of 256-byte rows
+    assert (a["threads"], a["unroll"], a["ctas_per_sm"], a["max_ctas"], a["debug_bounds"]) == (256, 4, 2, 0, 0)
+    assert a["vec_bytes"] == 32 and a["src_order"] == 0 and a["lc_skew"] == 0
+    assert (b["threads"], b["unroll"], b["ctas_per_sm"], b["lc_skew"], b["max_ctas"], b["debug_bounds"],
+            b["src_order"]) == (128, 2, 5, 8, 64, 1, 1)
+    assert B.pdkv_plan_option(tuned_plan, "threads") == 128 and B.pdkv_plan_option(default_plan, "threads") == 0
+    B.pdkv_tune("threads", 64)                  # later changes reach neither plan
+    try:
+        assert B.pdkv_plan_launch_shape(default_plan, B.PDKV_OP_TRANSFER, 0, L) == a
+        assert B.pdkv_plan_launch_shape(tuned_plan, B.PDKV_OP_TRANSFER, 0, L) == b
+    finally:
+        B.pdkv_tune("threads", before["threads"])
+    # a skew never exceeds the strips of the call: one layer has two
+    assert B.pdkv_plan_launch_shape(tuned_plan, B.PDKV_OP_TRANSFER, 1, 2)["lc_skew"] == 2
+    with pytest.raises(B.PdkvError):
+        B.pdkv_plan_launch_shape(tuned_plan, B.PDKV_OP_TRANSFER, 0, L + 1)
+    with pytest.raises(B.PdkvError):
+        B.pdkv_plan_option(tuned_plan, "no_such_key")
+    for p in (default_plan, tuned_plan):
+        B.pdkv_plan_destroy(p)
+    B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
+
+
+def test_chooser_classes_of_copy():
+    """The built-in launch choice per class of copy, read back without a GPU: flat copies,
+    row-permuting copies, the 70B-shaped stride that switches the strip skew on, rows that
+    are not whole 64-byte sector pairs (walked in read order), small tiles (thread groups)."""
+    def shapes(w):
+        ps, pd = _pools(w)
+        plan = _plan(w, ps, pd)
+        out = [B.pdkv_plan_launch_shape(plan, op, 0, w.src.num_layers) for op in range(3)]
+        B.pdkv_plan_destroy(plan); B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
+        return out
+
+    pack, unpack, fused = shapes(W.make_config(2, n_req=2))                   # block-major both sides: flat
+    assert all((s["threads"], s["unroll"], s["group_threads"]) == (512, 1, 512) for s in (pack, unpack, fused))
+    assert all(s["lc_skew"] == 0 and s["src_order"] == 0 for s in (pack, unpack, fused))
+    pack, unpack, fused = shapes(W.make_config(4, n_req=2))                   # 80 layers x 64 tokens: 5 x 4 MiB blocks
+    assert (pack["threads"], pack["unroll"]) == (512, 1) and (fused["threads"], fused["unroll"]) == (256, 4)
+    assert pack["lc_skew"] == 16 and fused["lc_skew"] == 16 and unpack["lc_skew"] == 0
+    assert pack["lc_skew_shift"] == 2                                          # four 32 KiB tiles per 128 KiB strip
+    pack, unpack, fused = shapes(W.make_config(3, n_req=4, head_dim=80))      # 160-byte rows
+    assert pack["src_order"] == 0 and unpack["src_order"] == 1 and fused["src_order"] == 1
+    assert all(s["vec_bytes"] == 32 for s in (pack, unpack, fused))
+    pack, unpack, fused = shapes(W.make_config(3, n_req=4, num_kv_heads=1))   # 4 KiB tiles: groups of threads
+    assert fused["group_threads"] < fused["threads"] and fused["group_threads"] % 32 == 0

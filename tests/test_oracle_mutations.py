@@ -16,7 +16,7 @@ import pytest
 sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
 sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
 from paper_2408_08147_b200 import workloads as W
-from test_oracle_pins import _golden_rows, numpy_pack, numpy_scatter, tiny_workload
+from test_oracle_pins import _golden_rows, numpy_pack, numpy_scatter, subranges_agree_with_numpy, tiny_workload
 
 ORACLE_DIR = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "oracle")
 SENT = W.SENTINEL_U16
@@ -51,6 +51,15 @@ MUTATIONS = {
     "unpack ignores the layer range":
         ("void okv_unpack(const okv_geom *dg, uint8_t *dst, const okv_batch *bt,\n                const uint8_t *buf, int l0, int l1, int r0, int r1)\n{",
          "void okv_unpack(const okv_geom *dg, uint8_t *dst, const okv_batch *bt,\n                const uint8_t *buf, int l0, int l1, int r0, int r1)\n{\n    l0 = 0; l1 = dg->L;"),
+    "fused transfer ignores the layer range":
+        ("                  uint8_t *dst, const okv_batch *bt, int l0, int l1, int r0, int r1)\n{\n    const int E = sg->E;",
+         "                  uint8_t *dst, const okv_batch *bt, int l0, int l1, int r0, int r1)\n{\n    const int E = sg->E;\n    l0 = 0; l1 = sg->L;"),
+    "pack ignores the request range":
+        ("              uint8_t *buf, int l0, int l1, int r0, int r1)\n{\n    const int E = sg->E;",
+         "              uint8_t *buf, int l0, int l1, int r0, int r1)\n{\n    const int E = sg->E;\n    r0 = 0; r1 = bt->n_req;"),
+    "unpack: tail zeroing ignores the request range":
+        ("        zero_tail(dg, dst, bt, r, l0, l1);\n    }\n}\n\n/* Blocks -> blocks",
+         "    }\n    for (int r = 0; r < bt->n_req; ++r)\n        zero_tail(dg, dst, bt, r, l0, l1);\n}\n\n/* Blocks -> blocks"),
 }
 
 
@@ -129,6 +138,14 @@ def battery(o) -> bool:
             rest = (slice(None), slice(1, None)) if w.dst.layout == W.BLOCK_MAJOR else (slice(1, None),)
             if not np.array_equal(g6[lay], w6[lay]) or not (g6[rest] == SENT).all():
                 return False
+        # layer and request sub-ranges of all three calls
+        L, R = w.src.num_layers, w.batch.n_req
+        l0 = int(rng.integers(0, L)); l1 = int(rng.integers(l0, L + 1))
+        r0 = int(rng.integers(0, R)); r1 = int(rng.integers(r0, R + 1))
+        if not subranges_agree_with_numpy(o, w, s, l0, l1, r0, r1):
+            return False
+        if L > 1 and R > 1 and not subranges_agree_with_numpy(o, w, s, L - 1, L, R - 1, R):
+            return False
     return True
 
 

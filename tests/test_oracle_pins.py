@@ -353,6 +353,61 @@ def test_per_layer_equals_whole_model(oracle, seed):
     assert np.array_equal(d_whole, d_piece)
 
 
+def subranges_agree_with_numpy(o, w, src, l0, l1, r0, r1) -> bool:
+    """Layer range [l0,l1) and request range [r0,r1) of pack, unpack and the fused transfer
+    against the numpy restatement: exactly those layers of exactly those requests move, at
+    the offsets of a whole call; everything else keeps the sentinel."""
+    G = w.dst.block_tokens
+    L, HD = w.src.num_layers, w.src.num_kv_heads * w.src.head_dim
+    want_buf_all = numpy_pack(w, src)
+    n = want_buf_all.size
+    # per-request extents of the buffer from the numpy statement alone
+    sizes = [int(kept_mask(w.batch, r, G).sum()) * 2 * L * HD for r in range(w.batch.n_req)]
+    starts = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    want_buf = np.full(n, SENT, np.uint16)
+    for r in range(r0, r1):
+        per_layer = sizes[r] // L
+        a = starts[r] + l0 * per_layer
+        want_buf[a:a + (l1 - l0) * per_layer] = want_buf_all[a:a + (l1 - l0) * per_layer]
+    got_buf = np.full(n, SENT, np.uint16)
+    o.pack(w.src, src, w.batch, G, got_buf, layers=(l0, l1), requests=(r0, r1))
+    if not np.array_equal(got_buf, want_buf):
+        return False
+    # decode pool: the chosen requests alone, through the numpy scatter, then only the chosen layers
+    d0 = W.sentinel_pool_numpy(w.dst)
+    part = W.Workload(w.name, w.seed, w.src, w.dst, W.slice_batch(w.batch, r0, r1))
+    full = numpy_scatter(part, src, d0).reshape(w.dst.shape())
+    want = d0.copy().reshape(w.dst.shape())
+    if w.dst.layout == W.BLOCK_MAJOR:
+        want[:, l0:l1] = full[:, l0:l1]
+    else:
+        want[l0:l1] = full[l0:l1]
+    want = want.reshape(-1)
+    got = d0.copy()
+    o.unpack(w.dst, got, w.batch, want_buf_all, layers=(l0, l1), requests=(r0, r1))
+    if not np.array_equal(got, want):
+        return False
+    got = d0.copy()
+    o.transfer(w.src, src, w.dst, got, w.batch, layers=(l0, l1), requests=(r0, r1))
+    return bool(np.array_equal(got, want))
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_layer_and_request_subranges_against_numpy(oracle, seed):
+    rng = np.random.default_rng(4200 + seed)
+    w = tiny_workload(rng, skip=bool(seed % 2))
+    src = W.fill_pool_numpy(w.src, w.seed)
+    L, R = w.src.num_layers, w.batch.n_req
+    l0 = int(rng.integers(0, L))
+    l1 = int(rng.integers(l0, L + 1))
+    r0 = int(rng.integers(0, R))
+    r1 = int(rng.integers(r0, R + 1))
+    assert subranges_agree_with_numpy(oracle, w, src, l0, l1, r0, r1)
+    assert subranges_agree_with_numpy(oracle, w, src, 0, L, 0, R)
+    if L > 1 and R > 1:
+        assert subranges_agree_with_numpy(oracle, w, src, L - 1, L, R - 1, R)
+
+
 def test_threads_and_request_ranges_agree(oracle):
     w = W.make_config(5, num_layers=2, n_req=24)
     src = W.fill_pool_numpy(w.src, w.seed)

@@ -22,7 +22,7 @@ def _free_port():
         return s.getsockname()[1]
 
 
-def _worker(rank, port, idx, kw, chunk_blocks, q):
+def _worker(rank, port, idx, kw, chunk_blocks, q, layers_per_stage=0):
     os.environ.update(RANK=str(rank), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
     sys.path.insert(0, ROOT)
     import torch
@@ -52,15 +52,17 @@ def _worker(rank, port, idx, kw, chunk_blocks, q):
                 pool = B.pdkv_pool_create(B.desc_of(w.src), FAKE_BASE, w.src.num_bytes(), 0)
                 plan = B.pdkv_plan_create(pool, None, self.G, b.seq_len, b.src_tbl_off, b.src_tbl,
                                           meta.dst_tbl_off if meta.dst_skip is not None else None, None, meta.dst_skip)
-                self.buffer_bytes, self.offsets = B.pdkv_plan_buffer(plan, b.n_req)
+                self.buffer_bytes, self.request_offsets = B.pdkv_plan_buffer(plan, b.n_req)
+                self.num_layers = w.src.num_layers
                 B.pdkv_plan_destroy(plan)
                 B.pdkv_pool_destroy(pool)
 
-            def pack(self, buf):
+            def pack(self, buf, layers=None):
                 assert self.buffer_bytes == O.buffer_elems(self.batch, self.G, w.src) * w.src.elem_bytes
-                O.pack(w.src, src, self.batch, self.G, buf.numpy()[:self.buffer_bytes].view(np.uint16))
+                O.pack(w.src, src, self.batch, self.G, buf.numpy()[:self.buffer_bytes].view(np.uint16), layers=layers)
 
-        sent, _, _ = p2d.send_kv(b.seq_len, Sender, new_buffer, peer=1, chunk_bytes=chunk)
+        sent, _, _ = p2d.send_kv(b.seq_len, Sender, new_buffer, peer=1, chunk_bytes=chunk,
+                                 layers_per_stage=layers_per_stage)
         q.put(("sender", sent, True))
     else:                                  # receiver: decode pool, decode tables, resident-block mask
         dst = W.sentinel_pool_numpy(w.dst)
@@ -71,14 +73,18 @@ def _worker(rank, port, idx, kw, chunk_blocks, q):
                 self.batch = W.Batch(seq_len, np.zeros(b.n_req + 1, np.int64), z32, b.dst_tbl_off, b.dst_tbl, b.dst_skip)
                 pool = B.pdkv_pool_create(B.desc_of(w.dst), FAKE_BASE, w.dst.num_bytes(), 0)
                 plan = B.pdkv_plan_create(None, pool, G, seq_len, None, None, b.dst_tbl_off, b.dst_tbl, b.dst_skip)
-                self.buffer_bytes, self.offsets = B.pdkv_plan_buffer(plan, b.n_req)
+                self.buffer_bytes, self.request_offsets = B.pdkv_plan_buffer(plan, b.n_req)
+                self.num_layers = w.dst.num_layers
                 B.pdkv_plan_destroy(plan)
                 B.pdkv_pool_destroy(pool)
 
-            def unpack(self, buf):
-                O.unpack(w.dst, dst, self.batch, buf.numpy()[:self.buffer_bytes].view(np.uint16))
+            def unpack(self, buf, layers=None):
+                O.unpack(w.dst, dst, self.batch, buf.numpy()[:self.buffer_bytes].view(np.uint16), layers=layers)
 
-        got, _, _ = p2d.recv_kv(b.dst_tbl_off, b.dst_skip, G, Receiver, new_buffer, peer=0, chunk_bytes=chunk)
+        # the buffer starts as sentinel bytes, so a range that is restored before it has arrived shows
+        new_buffer = lambda n: torch.full((n,), 0xC1, dtype=torch.uint8)
+        got, _, _ = p2d.recv_kv(b.dst_tbl_off, b.dst_skip, G, Receiver, new_buffer, peer=0, chunk_bytes=chunk,
+                                layers_per_stage=layers_per_stage)
         want = W.sentinel_pool_numpy(w.dst)
         O.transfer(w.src, W.fill_pool_numpy(w.src, w.seed), w.dst, want, b)
         q.put(("receiver", got, bool(np.array_equal(dst, want))))
@@ -86,18 +92,20 @@ def _worker(rank, port, idx, kw, chunk_blocks, q):
     dist.destroy_process_group()
 
 
-@pytest.mark.parametrize("idx,kw,chunk_blocks", [
-    (3, dict(num_layers=2, n_req=6, max_len=700), 0),      # re-blocking 16 -> 128, the buffer as a whole
-    (5, dict(num_layers=2, n_req=24), 0),                  # resident blocks: the mask travels in the meta exchange
-    (5, dict(num_layers=2, n_req=24), 1),                  # the same bytes, one prefill block's worth per message
+@pytest.mark.parametrize("idx,kw,chunk_blocks,layers_per_stage", [
+    (3, dict(num_layers=2, n_req=6, max_len=700), 0, 0),   # re-blocking 16 -> 128, the buffer as a whole
+    (5, dict(num_layers=2, n_req=24), 0, 0),               # resident blocks: the mask travels in the meta exchange
+    (5, dict(num_layers=2, n_req=24), 1, 0),               # the same bytes, one prefill block's worth per message
+    (3, dict(num_layers=5, n_req=6, max_len=700), 0, 2),   # per-layer trigger: stages of 2, 2 and 1 layers
+    (5, dict(num_layers=3, n_req=24), 0, 1),               # one layer per stage; some requests are fully resident
 ])
-def test_two_rank_transfer_equals_single_process_transfer(idx, kw, chunk_blocks):
+def test_two_rank_transfer_equals_single_process_transfer(idx, kw, chunk_blocks, layers_per_stage):
     import torch.multiprocessing as mp
 
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
     port = _free_port()
-    procs = [ctx.Process(target=_worker, args=(r, port, idx, kw, chunk_blocks, q)) for r in range(2)]
+    procs = [ctx.Process(target=_worker, args=(r, port, idx, kw, chunk_blocks, q, layers_per_stage)) for r in range(2)]
     for p in procs:
         p.start()
     got = dict()
@@ -111,7 +119,7 @@ def test_two_rank_transfer_equals_single_process_transfer(idx, kw, chunk_blocks)
     assert got["receiver"][1], "the receiver's decode pool differs from a single-process transfer"
 
 
-def _gpu_worker(rank, port, idx, kw, q):
+def _gpu_worker(rank, port, idx, kw, q, layers_per_stage=0):
     os.environ.update(RANK=str(rank), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
     sys.path.insert(0, ROOT)
     import torch
@@ -130,7 +138,7 @@ def _gpu_worker(rank, port, idx, kw, q):
         src_t = torch.from_numpy(W.fill_pool_numpy(w.src, w.seed).view(np.uint8).copy()).cuda()
         torch.cuda.synchronize()
         sent, sess, _buf = p2d.send_kv(b.seq_len, p2d.gpu_sender(w.src, src_t, b.src_tbl_off, b.src_tbl, b.seq_len),
-                                       pinned, peer=1)
+                                       pinned, peer=1, layers_per_stage=layers_per_stage)
         sess.synchronize()
         sess.close()
         q.put(("sender", sent, True))
@@ -138,7 +146,8 @@ def _gpu_worker(rank, port, idx, kw, q):
         dst_t = torch.from_numpy(W.sentinel_pool_numpy(w.dst).view(np.uint8).copy()).cuda()
         torch.cuda.synchronize()
         got, sess, _buf = p2d.recv_kv(b.dst_tbl_off, b.dst_skip, w.dst.block_tokens,
-                                      p2d.gpu_receiver(w.dst, dst_t, b.dst_tbl_off, b.dst_tbl, b.dst_skip), pinned, peer=0)
+                                      p2d.gpu_receiver(w.dst, dst_t, b.dst_tbl_off, b.dst_tbl, b.dst_skip), pinned, peer=0,
+                                      layers_per_stage=layers_per_stage)
         sess.synchronize()
         sess.close()
         want = W.sentinel_pool_numpy(w.dst)
@@ -149,8 +158,11 @@ def _gpu_worker(rank, port, idx, kw, q):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("idx,kw", [(3, dict(num_layers=2, n_req=6, max_len=700)), (5, dict(num_layers=2, n_req=24))])
-def test_two_rank_transfer_with_the_library_kernels(idx, kw):
+@pytest.mark.parametrize("idx,kw,layers_per_stage", [(3, dict(num_layers=2, n_req=6, max_len=700), 0),
+                                                     (5, dict(num_layers=2, n_req=24), 0),
+                                                     (3, dict(num_layers=5, n_req=6, max_len=700), 2),
+                                                     (5, dict(num_layers=4, n_req=24), 1)])
+def test_two_rank_transfer_with_the_library_kernels(idx, kw, layers_per_stage):
     """The same protocol with the library on both ends: two processes that share
     the one GPU (their kernels never wait on each other), the contiguous buffer in
     pinned host memory on each side (the kernels write / read it over PCIe) and
@@ -163,7 +175,7 @@ def test_two_rank_transfer_with_the_library_kernels(idx, kw):
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
     port = _free_port()
-    procs = [ctx.Process(target=_gpu_worker, args=(r, port, idx, kw, q)) for r in range(2)]
+    procs = [ctx.Process(target=_gpu_worker, args=(r, port, idx, kw, q, layers_per_stage)) for r in range(2)]
     for p in procs:
         p.start()
     got = dict()
@@ -175,3 +187,33 @@ def test_two_rank_transfer_with_the_library_kernels(idx, kw):
         assert p.exitcode == 0
     assert got["sender"][0] == got["receiver"][0] > 0
     assert got["receiver"][1], "the receiver's decode pool differs from the checker's transfer"
+
+
+def test_stage_pieces_partition_the_buffer(oracle):
+    """The byte ranges a layer stage sends are exactly the layer ranges the checker's pack
+    writes for those layers, and over all stages they cover the buffer once."""
+    sys.path.insert(0, ROOT)
+    from paper_2408_08147_b200 import p2d
+    from paper_2408_08147_b200 import workloads as W
+
+    w = W.make_config(5, num_layers=5, n_req=30)
+    G, L = w.dst.block_tokens, w.src.num_layers
+    E = w.src.elem_bytes
+    off = oracle.request_offsets(w.batch, G, w.src) * E
+    assert (oracle.kept_tokens(w.batch, G) == 0).any()          # fully resident requests send nothing
+    src = W.fill_pool_numpy(w.src, w.seed)
+    n = oracle.buffer_elems(w.batch, G, w.src)
+    covered = np.zeros(n * E, np.int32)
+    assert p2d.layer_stages(L, 2) == [(0, 2), (2, 4), (4, 5)]
+    for l0, l1 in p2d.layer_stages(L, 2):
+        buf = np.full(n, W.SENTINEL_U16, np.uint16)
+        oracle.pack(w.src, src, w.batch, G, buf, layers=(l0, l1))
+        written = np.repeat(buf != W.SENTINEL_U16, E)
+        mask = np.zeros(n * E, bool)
+        for a, z in p2d.stage_pieces(off, L, l0, l1):
+            assert z > a
+            mask[a:z] = True
+            covered[a:z] += 1
+        assert np.array_equal(mask, written)
+    assert (covered == 1).all()
+    assert p2d.stage_pieces(off, L, 0, L) == [(0, n * E)]        # a whole-model stage is one message

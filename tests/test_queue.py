@@ -102,3 +102,42 @@ def test_queue_transfers_match_the_checker(oracle, host_pools):
     got = h_dst.numpy().view(np.uint16) if host_pools else dst_t.cpu().numpy().view(np.uint16)
     assert np.array_equal(got, want)
     B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
+
+
+@pytest.mark.gpu
+def test_submit_waits_for_the_producer_of_the_blocks(oracle):
+    """The slot streams run beside the caller's streams.  Here the prefill pool is written on
+    another stream, behind a long-running kernel, and nothing synchronises on the host before
+    the submit: only the event handed to pdkv_queue_submit orders the transfer after it."""
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    B.pdkv_tune("dry_run", 0)
+    w = W.make_config(3, num_layers=2, n_req=6, max_len=800)
+    src = W.fill_pool_numpy(w.src, w.seed)
+    sent = W.sentinel_pool_numpy(w.dst)
+    want = sent.copy()
+    oracle.transfer(w.src, src, w.dst, want, w.batch)
+    staged = torch.from_numpy(src.view(np.uint8).copy()).cuda()       # the values the producer will write
+    src_t = torch.zeros_like(staged)                                   # the pool starts out stale
+    dst_t = torch.from_numpy(sent.view(np.uint8).copy()).cuda()
+    ballast = torch.empty(1 << 28, dtype=torch.float32, device="cuda")
+    ps = B.pdkv_pool_create(B.desc_of(w.src), src_t.data_ptr(), src_t.numel(), 0)
+    pd = B.pdkv_pool_create(B.desc_of(w.dst), dst_t.data_ptr(), dst_t.numel(), 0)
+    q = B.pdkv_queue_create(ps, pd, 0, 1)
+    producer = torch.cuda.Stream()
+    ready = torch.cuda.Event()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(producer):
+        for _ in range(20):                    # some milliseconds of work ahead of the pool's fill
+            ballast.normal_()
+        src_t.copy_(staged)
+        ready.record(producer)
+    t = _submit(q, w.batch, wait_event=ready.cuda_event)               # no host synchronisation before this
+    assert t is not None
+    B.pdkv_queue_wait(q, t)
+    B.pdkv_queue_release(q, t)
+    B.pdkv_queue_destroy(q)
+    torch.cuda.synchronize()
+    assert np.array_equal(dst_t.cpu().numpy().view(np.uint16), want)
+    B.pdkv_pool_destroy(ps); B.pdkv_pool_destroy(pd)
