@@ -703,8 +703,11 @@ def _replay_on(graph, stream, torch):
 def overlap_arm(args):
     """Per-layer trigger (Sec. 3.5): layer l is transferred on a side stream as soon
     as a stand-in for layer l's compute (one bf16 GEMM on the main stream) has
-    finished, while layer l+1 computes.  Reports compute alone, transfer alone,
-    and both overlapped, for the register and the bulk-copy variants."""
+    finished, while layer l+1 computes.  Reports compute alone, transfer alone and
+    both overlapped -- how much of the transfer is hidden and by how much the compute
+    sequence itself is held up -- for the kernels sharing all SMs with the GEMM, for
+    plain device copies (no kernel), and for the transfer kernel on an SM partition
+    of its own (green contexts) with the GEMM on the remaining SMs."""
     import torch
 
     from paper_2408_08147_b200 import binding as B
@@ -714,6 +717,8 @@ def overlap_arm(args):
     B.lib()
     torch.cuda.set_device(0)
     kw = {"n_req": args.n_req} if args.n_req else {}
+    if args.layouts:
+        kw["src_layout"], kw["dst_layout"] = ("AB".index(args.layouts[0]), "AB".index(args.layouts[1]))
     w = W.make_config(args.config, **kw)
     src_t, dst_t = alloc_pools(w, torch)
     L = w.src.num_layers
@@ -723,55 +728,77 @@ def overlap_arm(args):
     c = torch.empty(n, n, device="cuda", dtype=torch.bfloat16)
     # the transfer stream gets the higher priority: its CTAs are placed as soon as
     # a compute CTA retires instead of after the whole compute grid
-    main, side = torch.cuda.Stream(), torch.cuda.Stream(priority=-1 if args.side_priority else 0)
+    plain_main, plain_side = torch.cuda.Stream(), torch.cuda.Stream(priority=-1 if args.side_priority else 0)
     torch.cuda.synchronize()
 
-    def timed(fn, reps):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    def timed(fn, reps, main, side):
+        """(whole sequence, main stream alone) in ms per repetition; the second is when the
+        compute sequence itself finished, whatever the side stream still had to do."""
+        e0, e_main, e1 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
         fn()
         torch.cuda.synchronize()
         e0.record(main)
+        side.wait_event(e0)
         for _ in range(reps):
             fn()
+        e_main.record(main)
         side_done = torch.cuda.Event()
         side_done.record(side)
         main.wait_event(side_done)
         e1.record(main)
         torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / reps
+        return e0.elapsed_time(e1) / reps, e0.elapsed_time(e_main) / reps
 
-    def compute_only():
-        with torch.cuda.stream(main):
-            for _ in range(L):
-                torch.matmul(a, b, out=c)
+    def compute_on(main):
+        def fn():
+            with torch.cuda.stream(main):
+                for _ in range(L):
+                    torch.matmul(a, b, out=c)
+        return fn
 
-    results = {}
-    modes = [("register copy, defaults", {"variant": 0}),
-             ("register copy on at most 64 SMs", {"variant": 0, "ctas_per_sm": 1, "threads": 1024, "unroll": 1,
-                                                  "max_ctas": 64}),
-             ("register copy on at most 32 SMs", {"variant": 0, "ctas_per_sm": 1, "threads": 1024, "unroll": 1,
-                                                  "max_ctas": 32}),
-             ("register copy, one warp per CTA (32 threads x 8 accesses), 4 CTAs/SM",
-              {"variant": 0, "ctas_per_sm": 4, "threads": 32, "unroll": 8, "group_threads": 32}),
+    same_blocks = w.src.layout == 0 and w.dst.layout == 0 and w.src.block_tokens == w.dst.block_tokens
+    modes = [("register copy, defaults", {"variant": 0}, None),
+             ("register copy on at most 32 SMs (grid cap only, SMs shared with the GEMM)",
+              {"variant": 0, "ctas_per_sm": 1, "threads": 1024, "unroll": 1, "max_ctas": 32}, None),
              ("register copy, two warps per CTA (64 threads x 4 accesses), 8 CTAs/SM",
-              {"variant": 0, "ctas_per_sm": 8, "threads": 64, "unroll": 4, "group_threads": 64}),
+              {"variant": 0, "ctas_per_sm": 8, "threads": 64, "unroll": 4, "group_threads": 64}, None),
              ("bulk copy (TMA), 8 KiB tiles x 2 stages x 8 CTAs/SM",
-              {"variant": 1, "tile_bytes": 8192, "stages": 2, "ctas_per_sm": 8}),
+              {"variant": 1, "tile_bytes": 8192, "stages": 2, "ctas_per_sm": 8}, None),
              ("bulk copy with tiled TMA loads, 16 KiB tiles x 4 stages x 3 CTAs/SM",
-              {"variant": 2, "tile_bytes": 16384, "stages": 4, "ctas_per_sm": 3}),
-             ("bulk copy with tiled TMA loads, 16 KiB tiles x 2 stages x 2 CTAs/SM",
-              {"variant": 2, "tile_bytes": 16384, "stages": 2, "ctas_per_sm": 2})]
+              {"variant": 2, "tile_bytes": 16384, "stages": 4, "ctas_per_sm": 3}, None)]
+    if same_blocks:
+        modes.append(("plain device copies, one per block and layer (no kernel)", {"variant": 0}, "copies"))
+    for sms in (args.partition_sms or []):
+        modes.append((f"register copy on an SM partition of its own ({sms} SMs asked for)",
+                      {"variant": 0, "ctas_per_sm": 2}, sms))
     defaults = {k: B.pdkv_tune_get(k) for k in ("variant", "ctas_per_sm", "threads", "unroll", "tile_bytes", "stages",
                                                 "max_ctas", "group_threads")}
-    t_compute = timed(compute_only, args.steps)
-    for name, tune in modes:
+    t_compute, _ = timed(compute_on(plain_main), args.steps, plain_main, plain_side)
+    results = {}
+    for name, tune, special in modes:
+        main, side, part = plain_main, plain_side, None
+        tune = dict(tune)
+        rec = {}
+        try:
+            if isinstance(special, int):
+                part = B.pdkv_sm_partition_create(0, special)
+                got_t, got_c = B.pdkv_sm_partition_info(part)
+                side = torch.cuda.ExternalStream(B.pdkv_sm_partition_stream(part, 0))
+                main = torch.cuda.ExternalStream(B.pdkv_sm_partition_stream(part, 1))
+                tune["max_ctas"] = got_t * tune["ctas_per_sm"]
+                rec["sm_partition"] = {"transfer_sms": got_t, "compute_sms": got_c}
+        except B.PdkvError as e:
+            results[name] = {"unavailable": str(e)}
+            continue
         for k, v in {**defaults, **tune}.items():
             B.pdkv_tune(k, v)
         sess = TransferSession(w.src, src_t, w.dst, dst_t, w.batch, side.cuda_stream)
+        move = (lambda l: B.pdkv_transfer_copies(sess.plan, l, l + 1, side.cuda_stream)) if special == "copies" else \
+            (lambda l: sess.transfer((l, l + 1), side.cuda_stream))
 
         def transfer_only():
             for l in range(L):
-                sess.transfer((l, l + 1), side.cuda_stream)
+                move(l)
 
         def overlapped():
             for l in range(L):
@@ -780,21 +807,32 @@ def overlap_arm(args):
                     ev = torch.cuda.Event()
                     ev.record(main)
                 side.wait_event(ev)
-                sess.transfer((l, l + 1), side.cuda_stream)
+                move(l)
 
-        t_x = timed(transfer_only, args.steps)
-        t_o = timed(overlapped, args.steps)
-        # the same per-layer sequence recorded once into a CUDA graph and replayed
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=side):
-            cur = torch.cuda.current_stream().cuda_stream
-            for l in range(L):
-                sess.transfer((l, l + 1), cur)
-        t_g = timed(lambda: _replay_on(graph, side, torch), args.steps)
-        results[name] = {"transfer_alone_ms": t_x, "transfer_alone_graph_ms": t_g, "overlapped_ms": t_o,
-                         "serial_ms": t_compute + t_x,
-                         "hidden_fraction_of_transfer": max(0.0, min(1.0, (t_compute + t_x - t_o) / t_x))}
+        t_c, _ = timed(compute_on(main), args.steps, main, side) if part else (t_compute, None)
+        t_x, _ = timed(transfer_only, args.steps, main, side)
+        t_o, t_o_main = timed(overlapped, args.steps, main, side)
+        rec.update({"compute_alone_ms": t_c, "transfer_alone_ms": t_x, "overlapped_ms": t_o,
+                    "compute_sequence_while_overlapped_ms": t_o_main,
+                    "serial_ms": t_c + t_x,
+                    "hidden_fraction_of_transfer": max(0.0, min(1.0, (t_c + t_x - t_o) / t_x)),
+                    # how much longer the whole job takes than the GEMM sequence alone on the full GPU
+                    "job_slowdown_vs_compute_on_all_sms": t_o / t_compute - 1.0,
+                    "compute_slowdown_vs_all_sms": t_o_main / t_compute - 1.0})
+        if special is None:
+            # the same per-layer sequence recorded once into a CUDA graph and replayed
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                cur = torch.cuda.current_stream().cuda_stream
+                for l in range(L):
+                    sess.transfer((l, l + 1), cur)
+            rec["transfer_alone_graph_ms"], _ = timed(lambda: _replay_on(graph, side, torch), args.steps, main, side)
+        results[name] = rec
         sess.close()
+        if part:
+            torch.cuda.synchronize()
+            del main, side
+            B.pdkv_sm_partition_destroy(part)
     for k, v in defaults.items():
         B.pdkv_tune(k, v)
     out = {"mode": "overlap", "config": {"workload": workload_name(w), "layers": L,
@@ -902,7 +940,9 @@ def p2d_arm(args):
 
     block_bytes = w.src.num_bytes() // w.src.num_blocks
     results = {}
-    for name, chunk in (("whole buffer", 0), ("one prefill block per message", block_bytes)):
+    stage = max(1, args.p2d_layers_per_stage)
+    for name, chunk, lps in (("whole buffer", 0, 0), ("one prefill block per message", block_bytes, 0),
+                             (f"layer pipeline, {stage} layers per stage (pack | send | unpack overlap)", 0, stage)):
         times, nbytes = [], 0
         for it in range(args.warmup + args.steps):
             barrier()
@@ -910,11 +950,11 @@ def p2d_arm(args):
             t0 = time.perf_counter()
             if rank == 0:
                 nbytes, sess, _ = p2d.send_kv(b.seq_len, p2d.gpu_sender(w.src, pool_t, b.src_tbl_off, b.src_tbl, b.seq_len),
-                                              buffer, peer=1, device=meta_dev, chunk_bytes=chunk)
+                                              buffer, peer=1, device=meta_dev, chunk_bytes=chunk, layers_per_stage=lps)
             else:
                 nbytes, sess, _ = p2d.recv_kv(b.dst_tbl_off, b.dst_skip, w.dst.block_tokens,
                                               p2d.gpu_receiver(w.dst, pool_t, b.dst_tbl_off, b.dst_tbl, b.dst_skip),
-                                              buffer, peer=0, device=meta_dev, chunk_bytes=chunk)
+                                              buffer, peer=0, device=meta_dev, chunk_bytes=chunk, layers_per_stage=lps)
             torch.cuda.synchronize()
             dt = (time.perf_counter() - t0) * 1e3
             sess.close()
@@ -923,11 +963,13 @@ def p2d_arm(args):
                 times.append(ms)
         results[name] = {"ms": statistics.fmean(times), "ms_best": min(times), "buffer_bytes": nbytes,
                          "link_GBps": nbytes / (statistics.fmean(times) * 1e-3) / 1e9,
-                         "messages": max(1, -(-nbytes // chunk)) if chunk else 1}
+                         "messages": max(1, -(-nbytes // chunk)) if chunk else
+                         (len(p2d.layer_stages(w.src.num_layers, lps)) * b.n_req if lps else 1)}
     if rank == 0:
         a, c = results["whole buffer"]["ms"], results["one prefill block per message"]["ms"]
+        pipe = [v["ms"] for k, v in results.items() if k.startswith("layer pipeline")][0]
         print(json.dumps({"mode": "p2d", "config": {"workload": workload_name(w)}, "variants": results,
-                          "time_saved_by_block_free": 1.0 - a / c,
+                          "time_saved_by_block_free": 1.0 - a / c, "time_saved_by_layer_pipeline_vs_whole_buffer": 1.0 - pipe / a,
                           "transport": "gloo, pinned host buffers" if host else "NCCL send/recv between two GPUs",
                           "includes": "meta exchange, plan, pack, send/recv, unpack; wall clock, max over ranks"}),
               flush=True)
@@ -962,7 +1004,10 @@ def parse():
     ap.add_argument("--p2d", action="store_true", help="two ranks, two GPUs: pack -> one NCCL send/recv -> unpack")
     ap.add_argument("--p2d-host-buffers", action="store_true",
                     help="with --p2d: contiguous buffer in pinned host memory, gloo transport; the two ranks may share one GPU")
+    ap.add_argument("--p2d-layers-per-stage", type=int, default=4, help="with --p2d: layers per stage of the pipelined variant")
     ap.add_argument("--gemm-n", type=int, default=4096)
+    ap.add_argument("--partition-sms", type=int, action="append",
+                    help="with --overlap: also run the transfer on an SM partition of this many SMs (repeatable)")
     ap.add_argument("--side-priority", type=int, default=1, help="1: transfer stream has high priority")
     ap.add_argument("--no-blockwise", action="store_true")
     ap.add_argument("--autotune", action="store_true", help="pdkv_plan_autotune before the timed steps (not the default run)")

@@ -281,6 +281,17 @@ int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
  * Same result as pdkv_transfer over all layers. */
 int pdkv_transfer_blockwise(const pdkv_plan *plan, void *stream);
 
+/* The fused transfer of layers [layer_begin, layer_end) issued as plain device copies
+ * (cudaMemcpyAsync per prefill block, 2-D copies and memsets for a partial last block)
+ * instead of a kernel, for plans whose two pools are both block-major with the same
+ * block size: there a block's layer range is one contiguous byte range on either side.
+ * Same decode pool image as pdkv_transfer().  Such copies may be served by the GPU's copy
+ * engines and then take no SM from kernels that run beside them -- the no-interference
+ * form of the per-layer trigger (Sec. 3.5) -- at the price of one host call per block,
+ * the control cost Sec. 2.3 describes.
+ * Errors: INVALID_ARG, GEOMETRY (other layouts or unequal block sizes), CUDA. */
+int pdkv_transfer_copies(const pdkv_plan *plan, int layer_begin, int layer_end, void *stream);
+
 /* Host-resident pools.  `host_src_pool` / `host_dst_pool` (host; pinned memory
  * makes the copies asynchronous) are byte images of the prefill / decode pool
  * with the pool's own geometry.  pdkv_upload_blocks() copies every prefill
@@ -340,6 +351,26 @@ int pdkv_queue_release(pdkv_queue *queue, int64_t ticket);
 int pdkv_queue_stats(const pdkv_queue *queue, int *capacity, int *in_use, int64_t *submitted,
                      int64_t *rejected);
 int pdkv_queue_destroy(pdkv_queue *queue);
+
+/* SM partition for the per-layer trigger (Sec. 3.5: the transfer of layer l runs while
+ * layer l+1 computes, and as an operator it must not hold the other operators up).
+ * pdkv_sm_partition_create() splits the SMs of `device` into a transfer share of
+ * about `transfer_sms` (the driver rounds it up to its granularity, 8 on sm_90 and
+ * later) and the rest, as two CUDA green contexts of this process, each with one
+ * non-blocking stream: kernels enqueued on stream 0 (`which` = 0) run only on the
+ * transfer SMs, kernels on stream 1 only on the others, so neither waits for a CTA
+ * slot of the other.  Streams belong to the partition; use them like any
+ * cudaStream_t (for pdkv_transfer create the plan with "max_ctas" =
+ * transfer SMs x "ctas_per_sm", so that the persistent grid matches its share).
+ * Nothing outlasts the process and no device setting changes.  (No counterpart in
+ * the paper, whose transfer engine is not the compute device.)
+ * Errors: INVALID_ARG, NOMEM, CUDA (driver without green contexts, or a split the
+ * device refuses). */
+typedef struct pdkv_sm_partition pdkv_sm_partition;
+int pdkv_sm_partition_create(int device, int transfer_sms, pdkv_sm_partition **out);
+int pdkv_sm_partition_info(const pdkv_sm_partition *partition, int *transfer_sms, int *compute_sms);
+int pdkv_sm_partition_stream(const pdkv_sm_partition *partition, int which, void **stream);
+int pdkv_sm_partition_destroy(pdkv_sm_partition *partition);
 
 /* Number of GPU operations (kernel launches + memcpys) one call of `op`
  * enqueues; op = 3 asks about pdkv_transfer_blockwise. */
@@ -419,21 +450,27 @@ int pdkv_plan_option(const pdkv_plan *plan, const char *key, int64_t *value);
  *   "src_order"      order in which the threads of a CTA walk the rows of a tile whose
  *                    two sides differ in order (one token-major, one head-major): 0 in
  *                    the order of the side written, 1 of the side read, -1 (default)
- *                    automatic: read order when a row (D*E bytes) is not a multiple of
- *                    64 bytes -- a lone read of such a row fetches a sector more than it
- *                    uses -- else write order
+ *                    automatic: read order unless a row (D*E bytes) is a multiple of 256
+ *                    bytes (measured: lone reads of other row sizes cost 3-13%, and rows that
+ *                    are not whole 64-byte sector pairs fetch more DRAM bytes than they use)
  *   "debug_bounds"   1: kernels range-check every access and skip bad ones
  *   "debug_shrink"   with "debug_bounds": pretend each side is N bytes shorter, so
  *                    that the refusal path can be exercised on valid memory
- *   "variant"        0: register copy (default); 1: bulk async copies (TMA) through
- *                    shared memory, one warp per CTA; used when rows are multiples
- *                    of 16 bytes and a tile fits a stage, else variant 0 runs;
- *                    2: as 1, and tiles whose two sides differ in order (one
- *                    token-major, one head-major) are moved with tiled TMA loads
- *                    or stores through a tensor map of the token-major side (one
- *                    per head instead of one bulk copy per row) when the
- *                    geometry meets the TMA rules
- *   "stages"         variant 1: shared-memory stages per CTA, 2..16 (default 3);
+ *   "variant"        kernel family.  -1 (default): chosen per call -- the register copy (0),
+ *                    except that tiles going from a token-major side to a head-major one in
+ *                    rows of more than 128 bytes that are not multiples of 256, 24 KiB or more
+ *                    per tile, run the staged transpose (3).  0: register copy.  1: bulk async copies (TMA)
+ *                    through shared memory, one warp per CTA; used when rows are multiples
+ *                    of 16 bytes and a tile fits a stage, else variant 0 runs.  2: as 1, and
+ *                    tiles whose two sides differ in order (one token-major, one head-major)
+ *                    are moved with tiled TMA loads or stores through a tensor map of the
+ *                    token-major side (one per head instead of one bulk copy per row) when
+ *                    the geometry meets the TMA rules.  3: staged transpose for tiles whose
+ *                    two sides differ in order: bulk loads (TMA) fetch the tile in the order
+ *                    of the side that is read into a ring of shared-memory stages, all
+ *                    threads of the CTA store it in the order of the side that is written,
+ *                    so both sides see contiguous runs; other tiles run variant 0
+ *   "stages"         variants 1 to 3: shared-memory stages per CTA, 2..16 (default 3);
  *                    stages x "tile_bytes" must fit in 220 KiB
  *   "autotune_reuse" 1 (default): a new plan starts with the shapes that an earlier
  *                    pdkv_plan_autotune() found for the same geometry

@@ -44,6 +44,8 @@ EXPORTS = (
     "pdkv_queue_create", "pdkv_queue_submit", "pdkv_queue_poll", "pdkv_queue_wait", "pdkv_queue_release",
     "pdkv_queue_stats", "pdkv_queue_destroy", "pdkv_tune", "pdkv_tune_get", "pdkv_strerror",
     "pdkv_plan_autotune", "pdkv_plan_shape", "pdkv_plan_set_shape", "pdkv_plan_launch_shape", "pdkv_plan_option",
+    "pdkv_sm_partition_create", "pdkv_sm_partition_info", "pdkv_sm_partition_stream", "pdkv_sm_partition_destroy",
+    "pdkv_transfer_copies",
 )
 
 
@@ -118,6 +120,11 @@ def lib() -> C.CDLL:
     L.pdkv_queue_submit.argtypes = [vp, C.POINTER(pdkv_batch_desc), vp, vp, vp, C.POINTER(i64)]
     L.pdkv_plan_launch_shape.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.POINTER(pdkv_launch_shape)]
     L.pdkv_plan_option.argtypes = [vp, C.c_char_p, C.POINTER(i64)]
+    L.pdkv_sm_partition_create.argtypes = [C.c_int, C.c_int, C.POINTER(vp)]
+    L.pdkv_sm_partition_info.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+    L.pdkv_sm_partition_stream.argtypes = [vp, C.c_int, C.POINTER(vp)]
+    L.pdkv_sm_partition_destroy.argtypes = [vp]
+    L.pdkv_transfer_copies.argtypes = [vp, C.c_int, C.c_int, vp]
     L.pdkv_queue_poll.argtypes = [vp, i64, C.POINTER(C.c_int)]
     L.pdkv_queue_wait.argtypes = [vp, i64]
     L.pdkv_queue_release.argtypes = [vp, i64]
@@ -296,6 +303,34 @@ def pdkv_transfer_noalloc(src_pool: int, dst_pool: int, seq_len, src_tbl_off, sr
     _check(lib().pdkv_transfer_noalloc(C.c_void_p(src_pool), C.c_void_p(dst_pool), C.byref(b.desc),
                                        layer_begin, layer_end, C.c_void_p(stream)),
            "pdkv_transfer_noalloc")
+
+
+def pdkv_transfer_copies(plan: int, layer_begin: int, layer_end: int, stream: int = 0) -> None:
+    _check(lib().pdkv_transfer_copies(C.c_void_p(plan), layer_begin, layer_end, C.c_void_p(stream)),
+           "pdkv_transfer_copies")
+
+
+def pdkv_sm_partition_create(device: int, transfer_sms: int) -> int:
+    out = C.c_void_p()
+    _check(lib().pdkv_sm_partition_create(device, transfer_sms, C.byref(out)), "pdkv_sm_partition_create")
+    return out.value
+
+
+def pdkv_sm_partition_info(partition: int):
+    """(transfer SMs, compute SMs) as the driver rounded them."""
+    a, b = C.c_int(), C.c_int()
+    _check(lib().pdkv_sm_partition_info(C.c_void_p(partition), C.byref(a), C.byref(b)), "pdkv_sm_partition_info")
+    return a.value, b.value
+
+
+def pdkv_sm_partition_stream(partition: int, which: int) -> int:
+    out = C.c_void_p()
+    _check(lib().pdkv_sm_partition_stream(C.c_void_p(partition), which, C.byref(out)), "pdkv_sm_partition_stream")
+    return out.value
+
+
+def pdkv_sm_partition_destroy(partition: int) -> None:
+    _check(lib().pdkv_sm_partition_destroy(C.c_void_p(partition)), "pdkv_sm_partition_destroy")
 
 
 def pdkv_transfer_blockwise(plan: int, stream: int = 0) -> None:

@@ -76,6 +76,7 @@ struct pdkv_plan {
     std::vector<Tile> tiles[3];
     const Tile *dev_tiles[3] = {nullptr, nullptr, nullptr};
     std::vector<BlockGroup> groups;
+    bool same_blocks = false;   // both pools block-major with equal block size: a block's layer range is one byte range
     // maximal runs of consecutive block ids: prefill blocks the batch reads, decode blocks it writes
     std::vector<std::pair<int64_t, int64_t>> src_runs, dst_runs;  // (first id, count)
     void *dev_mem = nullptr;
@@ -89,7 +90,8 @@ struct pdkv_plan {
     // launch shape found by pdkv_plan_autotune() for each operation; threads == 0: not tuned
     struct Shape {
         int threads = 0, unroll = 0, ctas_per_sm = 0;
-        int skew = -1;   // strip skew: -1 by the stride rule, 0 none, > 0 this many strips
+        int skew = -1;      // strip skew: -1 by the stride rule, 0 none, > 0 this many strips
+        int variant = -1;   // kernel: -1 by the built-in rule, 0 register copy, 3 staged transpose
     } shape[3];
 };
 
@@ -155,6 +157,7 @@ void build_tiles(pdkv_plan &pl, int op, const pdkv_batch_desc &b, int64_t cap_to
     }
     const bool same_blocks = want_groups && pl.src.d.layout == PDKV_LAYOUT_BLOCK_MAJOR &&
                              pl.dst.d.layout == PDKV_LAYOUT_BLOCK_MAJOR && Bp == Bd;
+    if (want_groups) pl.same_blocks = same_blocks;
     for (int32_t r = 0; r < pl.n_req; ++r) {
         const int64_t len = b.seq_len[r];
         const uint8_t *skip = b.dst_skip ? b.dst_skip + b.dst_tbl_off[r] : nullptr;
@@ -272,7 +275,9 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     p.group_threads = 0;
     p.status = pl->dev_status;
     cudaError_t e;
-    if (r.cfg.variant >= 1 && pdkv::bulk_supported(r.cfg, p.row_bytes)) {
+    if (r.cfg.variant == 3 && pdkv::staged_supported(p, r.cfg)) {
+        e = pdkv::launch_staged(p, r.cfg, stream);
+    } else if ((r.cfg.variant == 1 || r.cfg.variant == 2) && pdkv::bulk_supported(r.cfg, p.row_bytes)) {
         r.cfg.vec_bytes = 16;
         e = pdkv::launch_bulk(p, r.cfg, stream);
     } else {
@@ -419,6 +424,7 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
         out->lc_skew_shift = (int32_t)shift;
     }
     LaunchConfig &cfg = out->cfg;
+    cfg.group_threads = 0;
     cfg.vec_bytes = pl->vec_bytes;
     if (pl->vec_bytes == 16 && o.vec32 && pl->row_bytes % 32 == 0 &&
         ((reinterpret_cast<uintptr_t>(src.base) | reinterpret_cast<uintptr_t>(dst.base)) & 31u) == 0)
@@ -428,19 +434,32 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
     cfg.ctas_per_sm = o.ctas_per_sm;
     cfg.max_ctas = o.max_ctas;
     cfg.sm_count = sm_count;
-    cfg.variant = o.variant;
     cfg.elem_bytes = pl->E;
     cfg.check_bounds = o.debug_bounds != 0;
     const int64_t hrow = pl->hrow_bytes, row = pl->row_bytes;
     const bool flat = src.head_stride == row && src.tok_stride == hrow && dst.head_stride == row &&
                       dst.tok_stride == hrow;
+    const bool small = pl->mean_tile_bytes[op] < 24 * 1024;
+    {   // Kernel.  Automatic: the register copy, except for tiles that go from a token-major side to
+        // a head-major one in rows of more than 128 bytes that are not multiples of 256 (head sizes
+        // such as 80, 96 or 112 at 2 bytes): those run the staged transpose, whose reads and writes are both contiguous runs
+        // (measured on 8B- and 70B-shaped batches with 80 to 192 dims per head: +3 to +12% over the
+        // register copy for tiles of 24 KiB and more; for smaller tiles and for 256-byte rows the
+        // register copy stays ahead).  pdkv_plan_autotune() may have timed the other choice.
+        int variant = o.variant;
+        if (variant < 0) {
+            const bool tok_to_head = src.tok_stride >= src.head_stride && dst.tok_stride < dst.head_stride;
+            variant = (tok_to_head && row % 256 != 0 && row > 128 && row % 16 == 0 && !small) ? 3 : 0;
+            if (pl->shape[op].variant >= 0) variant = pl->shape[op].variant;
+        }
+        cfg.variant = variant;
+    }
     {   // Automatic launch shape, measured best per class of copy on B200.  Full tiles
         // (about 32 KiB): a flat copy (token-major on both sides) runs 512 threads with
         // one access in flight each, i.e. two passes per tile; a copy with a head-major
         // side runs 256 threads with four, i.e. one pass per tile.  Batches of small
         // tiles (few KV heads, short blocks): groups of threads that cover a tile in two
         // passes of one access each, 32 threads at least.
-        const bool small = pl->mean_tile_bytes[op] < 24 * 1024;
         const pdkv_plan::Shape &tuned = pl->shape[op];
         const bool use_tuned = tuned.threads > 0 && cfg.unroll == 0 && cfg.threads == 0;
         if (use_tuned) {   // found by pdkv_plan_autotune(): the whole CTA works on one tile
@@ -456,9 +475,14 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
             cfg.unroll = 4;
             cfg.threads = 256;
         }
+        if (cfg.variant == 3 && cfg.threads == 0) {   // staged transpose: 256 threads store what one warp's bulk loads fetched
+            cfg.threads = 256;
+            cfg.unroll = 4;
+            if (o.group_threads == 0) cfg.group_threads = 256;
+        }
         if (cfg.unroll == 0) cfg.unroll = (flat || small) ? 1 : 4;
         if (cfg.threads == 0) cfg.threads = (flat || small) ? 512 : 256;
-        cfg.group_threads = o.group_threads;
+        if (cfg.group_threads == 0 || cfg.variant != 3) cfg.group_threads = o.group_threads;
         if ((use_tuned || odd_tile) && cfg.group_threads == 0) cfg.group_threads = cfg.threads;
         if (cfg.group_threads == 0) {
             const int64_t vecs = std::max<int64_t>(1, pl->mean_tile_bytes[op] / cfg.vec_bytes);
@@ -468,9 +492,11 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
             cfg.group_threads = g;
         }
     }
-    // Row order inside a tile (see CopyParams::src_order): rows that are not whole 64-byte
-    // pairs of sectors are walked in the order of the side that is read.
-    out->src_order = o.src_order >= 0 ? o.src_order : ((!flat && row % 64 != 0) ? 1 : 0);
+    // Row order inside a tile of the register copy (see CopyParams::src_order).  Measured on
+    // transposing copies with rows of 128 to 384 bytes: walking the rows in the order of the side
+    // that is read is 3-13% faster for every row size except multiples of 256 bytes, where the
+    // order of the side that is written wins by 5%.
+    out->src_order = o.src_order >= 0 ? o.src_order : ((!flat && row % 256 != 0) ? 1 : 0);
     cfg.stages = o.stages;
     cfg.max_tile_bytes = pl->max_tile_bytes;
 }
@@ -817,6 +843,23 @@ int pdkv_plan_autotune(pdkv_plan *plan, void *buf, size_t buf_bytes, void *strea
             }
         }
         plan->shape[op] = best;
+        // the other kernel for tiles that are transposed on the way (register copy <-> staged transpose),
+        // with that kernel's own built-in shape
+        if (rc == PDKV_OK && plan->opt.variant < 0 && op != PDKV_OP_PACK && plan->has_dst &&
+            plan->dst.d.layout == PDKV_LAYOUT_LAYER_MAJOR && (op == PDKV_OP_UNPACK || plan->src.d.layout == PDKV_LAYOUT_BLOCK_MAJOR) &&
+            plan->row_bytes % 16 == 0) {
+            const bool rule_staged = plan->row_bytes % 256 != 0 && plan->row_bytes > 128 && plan->mean_tile_bytes[op] >= 24 * 1024;
+            pdkv_plan::Shape other;
+            other.variant = rule_staged ? 0 : 3;
+            plan->shape[op] = other;
+            float ms = 0.f;
+            rc = time_ms(op, &ms);
+            if (rc == PDKV_OK && ms < 0.975f * best_ms) {
+                best_ms = ms;
+                best = other;
+            }
+            plan->shape[op] = best;
+        }
         // the strip skew the other way round: on where the stride rule leaves it off, off where it is on
         if (rc == PDKV_OK && plan->opt.lc_skew < 0 && plan->opt.lc_fastest == 0) {
             const pdkv_pool *pools[2] = {op != PDKV_OP_UNPACK && plan->has_src ? &plan->src : nullptr,
@@ -1031,6 +1074,39 @@ int pdkv_transfer_blockwise(const pdkv_plan *plan, void *stream)
     return PDKV_OK;
 }
 
+int pdkv_transfer_copies(const pdkv_plan *plan, int l0, int l1, void *stream)
+{
+    if (!plan || !plan->has_src || !plan->has_dst || !plan->dev_mem || !layers_ok(plan, l0, l1))
+        return PDKV_ERR_INVALID_ARG;
+    if (!plan->same_blocks) return PDKV_ERR_GEOMETRY;
+    if (l0 == l1) return PDKV_OK;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err, "cudaSetDevice");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t strip = (size_t)plan->src.d.block_tokens * (size_t)plan->hrow_bytes;   // one (layer, K/V) of a block
+    const size_t first = (size_t)2 * l0 * strip, n_lc = (size_t)2 * (l1 - l0);
+    const std::vector<Tile> &tiles = plan->tiles[PDKV_OP_TRANSFER];
+    for (const BlockGroup &g : plan->groups) {
+        cudaError_t e = cudaSuccess;
+        if (g.memcpy_bytes > 0) {   // a full block: its layers [l0, l1) are one contiguous range on both sides
+            e = cudaMemcpyAsync(plan->dst.base + g.memcpy_dst + first, plan->src.base + g.memcpy_src + first,
+                                n_lc * strip, cudaMemcpyDeviceToDevice, st);
+        } else {                    // a partial block: the valid tokens of each strip, then zeros for the rest
+            for (int32_t i = g.tile_begin; i < g.tile_end && e == cudaSuccess; ++i) {
+                const Tile &t = tiles[(size_t)i];
+                const size_t width = (size_t)t.ntok * (size_t)plan->hrow_bytes;
+                if (t.src_off >= 0)
+                    e = cudaMemcpy2DAsync(plan->dst.base + t.dst_off + first, strip, plan->src.base + t.src_off + first, strip,
+                                          width, n_lc, cudaMemcpyDeviceToDevice, st);
+                else
+                    e = cudaMemset2DAsync(plan->dst.base + t.dst_off + first, strip, 0, width, n_lc, st);
+            }
+        }
+        if (e != cudaSuccess) return cuda_fail(e, "block copy");
+    }
+    return PDKV_OK;
+}
+
 namespace {
 
 // Copy whole blocks between a host image of a pool and the device pool, one
@@ -1154,7 +1230,7 @@ int pdkv_tune(const char *key, int64_t value)
     else if (k == "group_threads" && (value == 0 || (value >= 32 && value <= 1024 && value % 32 == 0))) t.group_threads = value;
     else if (k == "debug_bounds" && (value == 0 || value == 1)) t.debug_bounds = value;
     else if (k == "debug_shrink" && value >= 0) t.debug_shrink = value;
-    else if (k == "variant" && value >= 0 && value <= 2) t.variant = value;
+    else if (k == "variant" && value >= -1 && value <= 3) t.variant = value;
     else if (k == "stages" && value >= 2 && value <= 16) t.stages = value;
     else if (k == "dry_run" && (value == 0 || value == 1)) t.dry_run = value;
     else if (k == "autotune_reuse" && (value == 0 || value == 1)) t.autotune_reuse = value;

@@ -109,6 +109,31 @@ struct Item {
     bool zero;
 };
 
+// Vector type of the staged kernel's stores: 16 bytes (one shared-memory load) or 32 (two).
+template <int W> struct StoreVec;
+template <> struct StoreVec<16> {
+    using type = uint4;
+    static __device__ __forceinline__ uint4 zero() { return make_uint4(0, 0, 0, 0); }
+    static __device__ __forceinline__ uint4 load_shared(const unsigned char *s) { return *reinterpret_cast<const uint4 *>(s); }
+    static __device__ __forceinline__ void store_global(char *g, const uint4 &v) { __stcs(reinterpret_cast<uint4 *>(g), v); }
+};
+template <> struct StoreVec<32> {
+    struct type {
+        uint4 lo, hi;
+    };
+    static __device__ __forceinline__ type zero() { return {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)}; }
+    static __device__ __forceinline__ type load_shared(const unsigned char *s)
+    {
+        return {*reinterpret_cast<const uint4 *>(s), *reinterpret_cast<const uint4 *>(s + 16)};
+    }
+    static __device__ __forceinline__ void store_global(char *g, const type &v)
+    {
+        asm volatile("st.global.cs.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};" ::"r"(v.lo.x), "r"(v.lo.y), "r"(v.lo.z),
+                     "r"(v.lo.w), "r"(v.hi.x), "r"(v.hi.y), "r"(v.hi.z), "r"(v.hi.w), "l"(g)
+                     : "memory");
+    }
+};
+
 }  // namespace
 
 __global__ void __launch_bounds__(32)
@@ -308,6 +333,157 @@ bulk_tiles_kernel(const CopyParams p, const int stages, const uint32_t stage_byt
     bulk_wait_all();
 }
 
+// "variant" 3: staged transpose.  For tiles whose two sides differ in order (one token-major,
+// one head-major) the tile is fetched in the order of the side that is READ -- one bulk copy of
+// the whole contiguous [token][head][dim] strip when that side is token-major, one contiguous
+// run per head when it is head-major -- into a ring of shared-memory stages, and all threads of
+// the CTA then write it out in the order of the side that is WRITTEN with coalesced vector stores
+// (consecutive lanes, consecutive addresses).  Neither side ever sees a lone row: every DRAM
+// sector pair that is fetched is used in full, whatever the row size (rows of 160 bytes read one
+// at a time fetch 192).  One mbarrier per stage counts the bytes of its loads; one
+// __syncthreads per tile hands the stage back.  Waits are bounded as in bulk_tiles_kernel.
+template <int W>
+__global__ void __launch_bounds__(512)
+staged_tiles_kernel(const CopyParams p, const int stages, const uint32_t stage_bytes)
+{
+    using V = typename StoreVec<W>::type;
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem);
+    unsigned char *data = smem + kBarrierBytes;
+    const uint32_t tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31u;
+    const uint32_t H = (uint32_t)p.H;
+    const uint32_t row = (uint32_t)p.row_bytes;
+    const uint32_t vpr = row / W;
+    const int64_t hrow = (int64_t)p.H * p.row_bytes;
+    const bool src_tok_major = p.src.tok_stride >= p.src.head_stride;   // the destination is the other way round
+    const uint32_t m_H = div_magic(H), m_vpr = div_magic(vpr);
+
+    if (tid == 0) {
+        for (int i = 0; i < stages; ++i) mbar_init(full + i, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    const int64_t n_work = (int64_t)p.n_tiles * p.n_lc;
+    int64_t first, step, n_mine;
+    if (p.chunked) {
+        const int64_t per = (n_work + gridDim.x - 1) / gridDim.x;
+        first = (int64_t)blockIdx.x * per;
+        const int64_t end = first + per < n_work ? first + per : n_work;
+        n_mine = end > first ? end - first : 0;
+        step = 1;
+    } else {
+        first = blockIdx.x;
+        step = gridDim.x;
+        n_mine = n_work > first ? (n_work - first + step - 1) / step : 0;
+    }
+
+    auto item = [&](int64_t j) {
+        const int64_t w = first + j * step;
+        int32_t ti, lci;
+        if (p.lc_fastest) {
+            ti = (int32_t)(w / p.n_lc);
+            lci = (int32_t)(w - (int64_t)ti * p.n_lc);
+        } else {
+            lci = (int32_t)(w / p.n_tiles);
+            ti = (int32_t)(w - (int64_t)lci * p.n_tiles);
+        }
+        if (p.lc_skew > 1) {   // as in the register-copy kernel: neighbouring tiles take different strips
+            lci += (ti >> p.lc_skew_shift) & (p.lc_skew - 1);
+            if (lci >= p.n_lc) lci -= p.n_lc;
+        }
+        const Tile t = p.tiles[p.tile_begin + ti];
+        const int64_t lc = p.lc_begin + lci;
+        const int64_t buf_lc = (int64_t)t.n_kept * hrow;
+        Item it;
+        it.s_base = t.src_off + lc * (p.src.lc_stride >= 0 ? p.src.lc_stride : buf_lc);
+        it.d_base = t.dst_off + lc * (p.dst.lc_stride >= 0 ? p.dst.lc_stride : buf_lc);
+        it.ntok = (uint32_t)t.ntok;
+        it.zero = t.src_off < 0;
+        return it;
+    };
+
+    // Warp 0 fills stage (j % stages) with item j in the order of the source.
+    auto issue_load = [&](int64_t j) {
+        const Item it = item(j);
+        uint64_t *bar = full + (j % stages);
+        unsigned char *st = data + (size_t)(j % stages) * stage_bytes;
+        if (it.zero) {                      // nothing to fetch: the stores write zeros
+            if (lane == 0) mbar_arrive(bar);
+            return;
+        }
+        if (lane == 0) mbar_arrive_expect(bar, it.ntok * H * row);
+        __syncwarp();
+        const char *src = p.src.base + it.s_base;
+        if (src_tok_major) {                // the tile is one contiguous strip of the source
+            if (lane == 0) bulk_g2s(st, src, it.ntok * H * row, bar);
+        } else {                            // one contiguous run of ntok rows per head
+            const uint32_t run = it.ntok * row;
+            for (uint32_t hd = lane; hd < H; hd += 32) bulk_g2s(st + (size_t)hd * run, src + hd * p.src.head_stride, run, bar);
+        }
+    };
+
+    int64_t head = 0;
+    for (int64_t tail = 0; tail < n_mine; ++tail) {
+        if (tid < 32) {                     // the stages being refilled were handed back at the last barrier
+            while (head < n_mine && head < tail + stages) {
+                issue_load(head);
+                ++head;
+            }
+        }
+        const Item it = item(tail);
+        const unsigned char *st = data + (size_t)(tail % stages) * stage_bytes;
+        uint32_t spins = 0;
+        bool ok = true;
+        while (!mbar_try_wait(full + (tail % stages), (uint32_t)((tail / stages) & 1))) {
+            if (++spins > kSpinLimit) {
+                ok = false;
+                break;
+            }
+        }
+        if (ok) {
+            // vectors in the order of the destination: (head, token) towards a head-major side,
+            // (token, head) towards a token-major one; the stage holds the order of the source
+            char *dst = p.dst.base + it.d_base;
+            const uint32_t ntok = it.ntok;
+            const uint32_t nvec = ntok * H * vpr;
+            const uint32_t inner = src_tok_major ? ntok : H;
+            const uint32_t m_inner = src_tok_major ? div_magic(ntok) : m_H;
+            constexpr int U = 4;
+            for (uint32_t i0 = tid; i0 < nvec; i0 += nthr * U) {
+                V v[U];
+                int64_t doff[U];
+#pragma unroll
+                for (int k = 0; k < U; ++k) {
+                    const uint32_t i = i0 + k * nthr;
+                    doff[k] = -1;
+                    if (i < nvec) {
+                        const uint32_t r = fast_div(i, m_vpr), vv = i - r * vpr;
+                        const uint32_t o = fast_div(r, m_inner), in = r - o * inner;
+                        const uint32_t hd = src_tok_major ? o : in, tk = src_tok_major ? in : o;
+                        const uint32_t soff = (src_tok_major ? tk * H + hd : hd * ntok + tk) * row + vv * W;
+                        doff[k] = tk * p.dst.tok_stride + hd * p.dst.head_stride + (int64_t)vv * W;
+                        v[k] = it.zero ? StoreVec<W>::zero() : StoreVec<W>::load_shared(st + soff);
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < U; ++k)
+                    if (doff[k] >= 0) StoreVec<W>::store_global(dst + doff[k], v[k]);
+            }
+        }
+        // hands the stage back to warp 0, and makes the outcome of the wait CTA-wide
+        if (!__syncthreads_and(ok ? 1 : 0)) {
+            if (tid == 0 && atomicCAS(p.status, 0ull, 2ull) == 0ull) p.status[1] = (unsigned long long)tail;
+            if (tid < 32)                    // loads still aimed at our stages: bounded wait each
+                for (int64_t j = tail + 1; j < head; ++j) {
+                    uint32_t s2 = 0;
+                    while (!mbar_try_wait(full + (j % stages), (uint32_t)((j / stages) & 1)) && ++s2 <= kSpinLimit) {}
+                }
+            return;
+        }
+    }
+}
+
 namespace {
 
 using EncodeTiled = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -386,6 +562,46 @@ cudaError_t launch_bulk(const CopyParams &p, const LaunchConfig &cfg, cudaStream
     if (cfg.max_ctas > 0 && grid > cfg.max_ctas) grid = cfg.max_ctas;
     if (grid > n_work) grid = n_work;
     bulk_tiles_kernel<<<(unsigned)grid, 32, smem, stream>>>(p, stages, stage_bytes, map, map_tokens);
+    return cudaGetLastError();
+}
+
+// Staged transpose ("variant" 3): the two sides differ in order, the token-major one is a dense
+// [token][head][dim] array, the head-major one keeps the tokens of a head adjacent.
+bool staged_supported(const CopyParams &p, const LaunchConfig &cfg)
+{
+    const int64_t row = p.row_bytes, hrow = (int64_t)p.H * row;
+    const bool src_tok_major = p.src.tok_stride >= p.src.head_stride;
+    const bool dst_tok_major = p.dst.tok_stride >= p.dst.head_stride;
+    if (src_tok_major == dst_tok_major) return false;
+    const Side &tm = src_tok_major ? p.src : p.dst, &hm = src_tok_major ? p.dst : p.src;
+    const size_t smem = kBarrierBytes + (size_t)cfg.stages * ((cfg.max_tile_bytes + 127) / 128 * 128);
+    return row % 16 == 0 && tm.tok_stride == hrow && tm.head_stride == row && hm.tok_stride == row &&
+           cfg.max_tile_bytes > 0 && cfg.max_tile_bytes <= 131072 && smem <= 220 * 1024 && cfg.stages >= 2 &&
+           !cfg.check_bounds && ((reinterpret_cast<uintptr_t>(p.src.base) | reinterpret_cast<uintptr_t>(p.dst.base)) & 15u) == 0;
+}
+
+cudaError_t launch_staged(const CopyParams &p, const LaunchConfig &cfg, cudaStream_t stream)
+{
+    const int64_t n_work = (int64_t)p.n_tiles * p.n_lc;
+    if (n_work <= 0) return cudaSuccess;
+    const uint32_t stage_bytes = (uint32_t)((cfg.max_tile_bytes + 127) / 128 * 128);
+    const int stages = cfg.stages;
+    const size_t smem = kBarrierBytes + (size_t)stages * stage_bytes;
+    const bool wide = p.row_bytes % 32 == 0 &&
+                      ((reinterpret_cast<uintptr_t>(p.dst.base) | (uintptr_t)p.dst.head_stride | (uintptr_t)p.dst.tok_stride) & 31u) == 0;
+    auto kern = wide ? staged_tiles_kernel<32> : staged_tiles_kernel<16>;
+    int threads = cfg.threads < 64 ? 64 : (cfg.threads > 512 ? 512 : cfg.threads / 32 * 32);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int occ = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, threads, smem);
+    if (e != cudaSuccess) return e;
+    if (occ < 1) return cudaErrorInvalidConfiguration;
+    if (occ > cfg.ctas_per_sm) occ = cfg.ctas_per_sm;
+    int64_t grid = (int64_t)cfg.sm_count * occ;
+    if (cfg.max_ctas > 0 && grid > cfg.max_ctas) grid = cfg.max_ctas;
+    if (grid > n_work) grid = n_work;
+    kern<<<(unsigned)grid, threads, smem, stream>>>(p, stages, stage_bytes);
     return cudaGetLastError();
 }
 

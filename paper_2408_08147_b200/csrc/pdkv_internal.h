@@ -55,7 +55,7 @@ struct LaunchConfig {
     int ctas_per_sm;
     int max_ctas;    // 0: no cap; else the grid is limited to this many CTAs (leaves SMs to other kernels)
     int sm_count;
-    int variant;             // 0 register copy, 1 bulk copies, 2 bulk copies with tiled TMA loads
+    int variant;             // 0 register copy, 1 bulk copies, 2 bulk copies with tiled TMA loads, 3 staged transpose
     int elem_bytes;          // element size, for the tensor map's data type
     int stages;              // bulk variant: shared-memory stages per CTA
     int64_t max_tile_bytes;  // bulk variant: largest tile of the launch
@@ -68,6 +68,9 @@ cudaError_t launch_copy(const CopyParams &p, const LaunchConfig &cfg, cudaStream
 // Bulk-copy (TMA) variant: same contract; bulk_supported() says whether a launch qualifies.
 cudaError_t launch_bulk(const CopyParams &p, const LaunchConfig &cfg, cudaStream_t stream);
 bool bulk_supported(const LaunchConfig &cfg, int row_bytes);
+// Staged transpose (bulk loads in read order, coalesced stores in write order): same contract.
+cudaError_t launch_staged(const CopyParams &p, const LaunchConfig &cfg, cudaStream_t stream);
+bool staged_supported(const CopyParams &p, const LaunchConfig &cfg);
 
 // Makes `dev` current for the lifetime of the object and restores the caller's device.
 struct DeviceGuard {
@@ -105,7 +108,7 @@ struct Tunables {
     std::atomic<int64_t> lc_skew_shift{0};
     std::atomic<int64_t> debug_bounds{0};
     std::atomic<int64_t> debug_shrink{0};   // with debug_bounds: treat the last N bytes of each side as out of range
-    std::atomic<int64_t> variant{0};
+    std::atomic<int64_t> variant{-1};   // -1: chosen per call (register copy or staged transpose)
     std::atomic<int64_t> stages{3};
     std::atomic<int64_t> dry_run{0};
     std::atomic<int64_t> autotune_reuse{1};
@@ -118,7 +121,7 @@ Tunables &tunables();
 // another thread).  pdkv_tune() only sets the defaults of plans created later.
 struct LaunchOptions {
     int ctas_per_sm = 2, max_ctas = 0, threads = 0, unroll = 0, vec32 = 1, lc_fastest = 0, group_threads = 0,
-        chunked = 0, lc_skew = -1, lc_skew_shift = 0, debug_bounds = 0, variant = 0, stages = 3, src_order = -1;
+        chunked = 0, lc_skew = -1, lc_skew_shift = 0, debug_bounds = 0, variant = -1, stages = 3, src_order = -1;
     int64_t debug_shrink = 0;
     int64_t tile_bytes = 32768;
 };

@@ -75,6 +75,11 @@ class TransferSession:
         l0, l1 = self._layers(layers)
         B.pdkv_transfer(self.plan, l0, l1, self.stream if stream is None else stream)
 
+    def transfer_copies(self, layers=None, stream: Optional[int] = None) -> None:
+        """The fused transfer as plain device copies (block-major pools of equal block size only)."""
+        l0, l1 = self._layers(layers)
+        B.pdkv_transfer_copies(self.plan, l0, l1, self.stream if stream is None else stream)
+
     def transfer_blockwise(self, stream: Optional[int] = None) -> None:
         B.pdkv_transfer_blockwise(self.plan, self.stream if stream is None else stream)
 

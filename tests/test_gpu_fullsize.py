@@ -31,13 +31,16 @@ def _defaults():
     torch.cuda.empty_cache()
 
 
-def _sentinel_fill(t):
-    t.view(torch.int16).fill_(SENT)
+# raw element types and "nobody may touch this" patterns per element size (the 1-byte pattern is
+# the one workloads.sentinel_pool_numpy uses)
+_TORCH_ELEM = {1: torch.uint8, 2: torch.int16}
+_NP_ELEM = {1: np.uint8, 2: np.uint16}
+_SENT = {1: 0xA5, 2: SENT}
+
+
+def _sentinel_fill(t, E=2):
+    t.view(_TORCH_ELEM[E]).fill_(_SENT[E])
     torch.cuda.synchronize()        # the library runs on its own stream
-
-
-def _np16(t):
-    return t.cpu().numpy().view(np.uint16)
 
 
 def _checksum(t):
@@ -52,8 +55,9 @@ class _Staging:
     """Pinned host buffers reused for every request group (pageable copies of
     tens of GiB would dominate the test's run time)."""
 
-    def __init__(self):
+    def __init__(self, E=2):
         self.bufs = {}
+        self.E = E
 
     def get(self, name, n_bytes):
         t = self.bufs.get(name)
@@ -65,13 +69,13 @@ class _Staging:
         h = self.get(name, dev_t.numel() * dev_t.element_size())
         h.copy_(dev_t.reshape(-1).view(torch.uint8))
         torch.cuda.synchronize()
-        return h.numpy().view(np.uint16)
+        return h.numpy().view(_NP_ELEM[self.E])
 
     def host_array(self, name, n_elems):
-        return self.get(name, 2 * n_elems).numpy().view(np.uint16)
+        return self.get(name, self.E * n_elems).numpy().view(_NP_ELEM[self.E])
 
     def to_device(self, name, n_elems):
-        return self.get(name, 2 * n_elems).cuda().view(torch.int16)
+        return self.get(name, self.E * n_elems).cuda().view(_TORCH_ELEM[self.E])
 
 
 def _checker_in_parallel(call, n_req, n_layers):
@@ -107,6 +111,8 @@ def run_fullsize(oracle, w, n_sample, seed, group=1):
     b = w.batch
     G = w.dst.block_tokens
     L = w.src.num_layers
+    E = w.src.elem_bytes
+    tdt, sent = _TORCH_ELEM[E], _SENT[E]
     payload = int(oracle.buffer_elems(b, G, w.src)) * w.src.elem_bytes
     free, _ = torch.cuda.mem_get_info()
     headroom = 12 << 30             # gathered sub-pools and torch's workspace
@@ -126,14 +132,14 @@ def run_fullsize(oracle, w, n_sample, seed, group=1):
     pools = [torch.empty(w.dst.num_bytes(), dtype=torch.uint8, device="cuda") for _ in range(n_pools)]
     stream = torch.cuda.Stream()
     torch.cuda.synchronize()
-    stage = _Staging()
+    stage = _Staging(E)
 
     sessions = [TransferSession(w.src, src_t, w.dst, p, b, stream.cuda_stream) for p in pools]
     try:
         s0 = sessions[0]
         assert s0.buffer_bytes == payload == sum(s0.traffic(B.PDKV_OP_PACK)) // 2
         buf_t = torch.empty(payload + SLACK, dtype=torch.uint8, device="cuda")
-        _sentinel_fill(buf_t)
+        _sentinel_fill(buf_t, E)
         calls = [("unpack", lambda s: (s.pack(buf_t), s.unpack(buf_t))),
                  ("fused", lambda s: s.transfer()),
                  ("block-by-block baseline", lambda s: s.transfer_blockwise())]
@@ -141,34 +147,34 @@ def run_fullsize(oracle, w, n_sample, seed, group=1):
         while calls:
             now, calls = calls[:n_pools], calls[n_pools:]
             for (what, call), s, pool in zip(now, sessions, pools):
-                _sentinel_fill(pool)
+                _sentinel_fill(pool, E)
                 call(s)
             torch.cuda.synchronize()
             for g in groups:
                 sub, s_ids, d_ids = W.compact_subproblem(w, g)
-                sub_src = stage.to_host("src", W.gather_blocks(src_t.view(torch.int16), w.src, s_ids))
+                sub_src = stage.to_host("src", W.gather_blocks(src_t.view(tdt), w.src, s_ids))
                 if first_pass:
                     want_buf = stage.host_array("buf", oracle.buffer_elems(sub.batch, G, sub.src))
                     want_buf[:] = 0
                     _checker_in_parallel(lambda **kw: oracle.pack(sub.src, sub_src, sub.batch, G, want_buf, **kw),
                                          len(g), L)
                     a, z = int(s0.request_offsets[g[0]]), int(s0.request_offsets[g[-1] + 1])
-                    assert want_buf.size * 2 == z - a
+                    assert want_buf.size * E == z - a
                     want_dev = stage.to_device("buf", want_buf.size)
-                    assert torch.equal(buf_t[a:z].view(torch.int16), want_dev), f"pack: requests {g[0]}..{g[-1]}"
+                    assert torch.equal(buf_t[a:z].view(tdt), want_dev), f"pack: requests {g[0]}..{g[-1]}"
                     del want_dev
                 want_dst = stage.host_array("dst", sub.dst.num_elems())
-                want_dst[:] = SENT
+                want_dst[:] = sent
                 _checker_in_parallel(lambda **kw: oracle.transfer(sub.src, sub_src, sub.dst, want_dst, sub.batch, **kw),
                                      len(g), L)
                 want_dev = stage.to_device("dst", want_dst.size)
                 for (what, _), pool in zip(now, pools):
-                    got = W.gather_blocks(pool.view(torch.int16), w.dst, d_ids)
+                    got = W.gather_blocks(pool.view(tdt), w.dst, d_ids)
                     assert torch.equal(got, want_dev), f"{what}: requests {g[0]}..{g[-1]}"
                     del got
                 del want_dev
             if first_pass:
-                assert bool((buf_t[payload:].view(torch.int16) == SENT).all()), "pack wrote past the buffer"
+                assert bool((buf_t[payload:].view(tdt) == sent).all()), "pack wrote past the buffer"
             # resident (skipped) decode blocks keep the sentinel after every call
             if b.dst_skip is not None:
                 nblk = -(-b.seq_len.astype(np.int64) // G)
@@ -178,8 +184,8 @@ def run_fullsize(oracle, w, n_sample, seed, group=1):
                 assert ids.size > 0
                 for (what, _), pool in zip(now, pools):
                     for i in range(0, ids.size, 64):
-                        blk = W.gather_blocks(pool.view(torch.int16), w.dst, ids[i:i + 64])
-                        assert bool((blk == SENT).all()), f"{what}: a resident decode block was written"
+                        blk = W.gather_blocks(pool.view(tdt), w.dst, ids[i:i + 64])
+                        assert bool((blk == sent).all()), f"{what}: a resident decode block was written"
             first_pass = False
         assert _checksum(src_t) == src_sum, "the prefill pool was written"
     finally:
@@ -210,3 +216,27 @@ def test_config4_full_size_70b_fragmented(oracle):
 @pytest.mark.parametrize("src_block", [16, 256])
 def test_config5_full_size_skip_mask(oracle, src_block):
     run_fullsize(oracle, W.make_config(5, src_block=src_block), n_sample=0, seed=5 + src_block, group=16)
+
+
+# Geometries beyond the five workloads as specified, at the sizes the benchmark times them:
+# few KV heads and 1-byte elements run the kernel instantiation in which a CTA is split into
+# independent thread groups (tiles of 2-16 KiB); 160-byte rows run the read-order walk.
+
+def test_config3_full_size_one_kv_head_one_byte_elements(oracle):
+    run_fullsize(oracle, W.make_config(3, num_kv_heads=1, elem_bytes=1), n_sample=0, seed=31, group=16)
+
+
+def test_config3_full_size_one_kv_head(oracle):
+    run_fullsize(oracle, W.make_config(3, num_kv_heads=1), n_sample=0, seed=32, group=16)
+
+
+def test_config2_full_size_one_byte_elements(oracle):
+    run_fullsize(oracle, W.make_config(2, elem_bytes=1), n_sample=0, seed=33, group=8)
+
+
+def test_config3_full_size_rows_of_160_bytes(oracle):
+    run_fullsize(oracle, W.make_config(3, head_dim=80), n_sample=0, seed=34, group=8)
+
+
+def test_config5_full_size_rows_of_160_bytes(oracle):
+    run_fullsize(oracle, W.make_config(5, head_dim=80), n_sample=0, seed=35, group=16)

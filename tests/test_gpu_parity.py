@@ -27,8 +27,9 @@ def _gpu_lib():
     B.pdkv_tune("lc_fastest", 0)
     B.pdkv_tune("lc_skew", -1)
     B.pdkv_tune("lc_skew_shift", 0)
-    B.pdkv_tune("variant", 0)
+    B.pdkv_tune("variant", -1)
     B.pdkv_tune("stages", 3)
+    B.pdkv_tune("src_order", -1)
 
 
 def dev(a: np.ndarray):
@@ -107,6 +108,8 @@ def test_config1_tiny_bounds_checked_then_plain(oracle):
     (5, dict(num_layers=2, n_req=24, src_block=256)),                    # prefill block > decode block
     (3, dict(num_layers=2, n_req=6, max_len=900, src_layout=W.LAYER_MAJOR,
              dst_layout=W.BLOCK_MAJOR)),                                 # B -> A
+    (3, dict(num_layers=2, n_req=10, max_len=1500, head_dim=80)),        # 160-byte rows
+    (5, dict(num_layers=2, n_req=30, head_dim=80)),                      # 160-byte rows, skip mask
 ])
 def test_scaled_configs(oracle, idx, kw):
     w = W.make_config(idx, **kw)
@@ -138,11 +141,12 @@ def test_tile_size_and_work_order_do_not_change_the_result(oracle, tile_bytes, l
         B.pdkv_tune("lc_skew_shift", 0)
 
 
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 @pytest.mark.parametrize("stages,tile_bytes,chunked", [(2, 16384, 0), (3, 65536, 0), (4, 32768, 1)])
 def test_bulk_copy_variant(oracle, variant, stages, tile_bytes, chunked):
     """Variants 1 and 2 (TMA bulk copies through a shared-memory ring; 2 adds tiled
-    tensor-map loads for the token-major -> head-major transpose) must produce the
+    tensor-map loads for the token-major -> head-major transpose) and 3 (bulk loads in
+    read order into shared memory, coalesced stores in write order) must produce the
     same bytes: flat, head-run and transposing tiles, ragged and zero-fill tiles,
     skip masks."""
     B.pdkv_tune("variant", variant)
@@ -163,11 +167,31 @@ def test_bulk_copy_variant(oracle, variant, stages, tile_bytes, chunked):
                              src_layout=W.BLOCK_MAJOR, src_block=7, dst_layout=W.LAYER_MAJOR, dst_block=5,
                              src_slack=1.3, dst_slack=1.3)
         check_all_ops(oracle, w)
+        # 160-byte rows (80 bf16) and 1-byte elements with 80-byte rows, both directions of the transpose
+        for lay in ((W.BLOCK_MAJOR, W.LAYER_MAJOR), (W.LAYER_MAJOR, W.BLOCK_MAJOR)):
+            check_all_ops(oracle, W.make_config(3, num_layers=2, n_req=6, max_len=700, head_dim=80, src_layout=lay[0],
+                                                dst_layout=lay[1]))
+        check_all_ops(oracle, W.make_config(5, num_layers=2, n_req=20, head_dim=80, elem_bytes=1), elem_dtype=np.uint8)
     finally:
-        B.pdkv_tune("variant", 0)
+        B.pdkv_tune("variant", -1)
         B.pdkv_tune("stages", 3)
         B.pdkv_tune("tile_bytes", 32768)
         B.pdkv_tune("chunked", 0)
+
+
+@pytest.mark.parametrize("src_order", [0, 1, -1])
+def test_row_order_inside_a_tile_does_not_change_the_result(oracle, src_order):
+    """Rows of a transposing tile are walked in the order of the side written (0), of the side
+    read (1), or chosen by the row size (-1: read order for 160-byte rows, write order for 256)."""
+    B.pdkv_tune("src_order", src_order)
+    try:
+        for D in (80, 128, 24):
+            check_all_ops(oracle, W.make_config(3, num_layers=2, n_req=6, max_len=800, head_dim=D))
+            check_all_ops(oracle, W.make_config(3, num_layers=2, n_req=5, max_len=600, head_dim=D,
+                                                src_layout=W.LAYER_MAJOR, dst_layout=W.BLOCK_MAJOR))
+        check_all_ops(oracle, W.make_config(5, num_layers=2, n_req=24, head_dim=80), layers=(1, 2))
+    finally:
+        B.pdkv_tune("src_order", -1)
 
 
 @pytest.mark.parametrize("seed", range(16))
@@ -511,3 +535,158 @@ def test_pinned_and_autotuned_launch_shapes(oracle):
                 assert all(B.pdkv_plan_shape(fresh.plan, op) == (0, 0, 0, -1) for op in ops)
     finally:
         B.pdkv_tune("autotune_reuse", 1)
+
+
+def test_transfer_as_plain_device_copies(oracle):
+    """Block-major pools with equal blocks: the fused transfer issued as device copies (one per
+    block and layer range, 2-D copies and memsets for partial blocks) writes the same bytes;
+    other geometries are refused."""
+    from paper_2408_08147_b200.session import TransferSession
+
+    for kw, layers in ((dict(num_layers=3, n_req=5, max_len=640), None), (dict(num_layers=4, n_req=4, max_len=333), (1, 3))):
+        w = W.make_config(2, **kw)
+        w.batch.seq_len[:] = np.array([kw["max_len"], 1, 129, 300, 256][:w.batch.n_req], np.int32)   # ragged tails
+        src = W.fill_pool_numpy(w.src, w.seed)
+        sent = W.sentinel_pool_numpy(w.dst)
+        want = sent.copy()
+        oracle.transfer(w.src, src, w.dst, want, w.batch, layers=layers)
+        src_t, dst_t = dev(src), dev(sent)
+        torch.cuda.synchronize()
+        with TransferSession(w.src, src_t, w.dst, dst_t, w.batch) as s:
+            s.transfer_copies(layers)
+            s.status()
+        assert np.array_equal(host(dst_t), want)
+    w = W.make_config(3, num_layers=2, n_req=3, max_len=300)            # re-blocking: not expressible as block copies
+    src_t, dst_t = dev(W.fill_pool_numpy(w.src, w.seed)), dev(W.sentinel_pool_numpy(w.dst))
+    with TransferSession(w.src, src_t, w.dst, dst_t, w.batch) as s:
+        with pytest.raises(B.PdkvError) as e:
+            s.transfer_copies()
+        assert e.value.status == B.PDKV_ERR_GEOMETRY
+
+
+@pytest.mark.parametrize("partition_sms", [0, 16])
+def test_per_layer_transfer_beside_a_compute_kernel(oracle, partition_sms):
+    """Sec. 3.5, per-layer trigger: layer l is transferred on a side stream while the main
+    stream computes (a matrix product stands in for layer l+1).  The decode pool must still
+    be bit-exact -- also when the transfer runs on an SM partition of its own."""
+    from paper_2408_08147_b200.session import TransferSession
+
+    w = W.make_config(3, num_layers=6, n_req=8, max_len=1200)
+    src = W.fill_pool_numpy(w.src, w.seed)
+    sent = W.sentinel_pool_numpy(w.dst)
+    want = sent.copy()
+    oracle.transfer(w.src, src, w.dst, want, w.batch)
+    src_t, dst_t = dev(src), dev(sent)
+    a = torch.randn(2048, 2048, device="cuda", dtype=torch.bfloat16)
+    c = torch.empty_like(a)
+    part = None
+    if partition_sms:
+        try:
+            part = B.pdkv_sm_partition_create(0, partition_sms)
+        except B.PdkvError as e:
+            pytest.skip(f"no SM partition on this driver: {e}")
+        t_sms, c_sms = B.pdkv_sm_partition_info(part)
+        assert t_sms >= partition_sms and c_sms > 0
+        total = torch.cuda.get_device_properties(0).multi_processor_count
+        assert t_sms + c_sms <= total
+        side = torch.cuda.ExternalStream(B.pdkv_sm_partition_stream(part, 0))
+        main = torch.cuda.ExternalStream(B.pdkv_sm_partition_stream(part, 1))
+        B.pdkv_tune("max_ctas", 2 * t_sms)
+    else:
+        main, side = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    try:
+        with TransferSession(w.src, src_t, w.dst, dst_t, w.batch, side.cuda_stream) as s:
+            if partition_sms:
+                assert B.pdkv_plan_launch_shape(s.plan, B.PDKV_OP_TRANSFER, 0, 1)["max_ctas"] == 2 * t_sms
+            for l in range(w.src.num_layers):
+                with torch.cuda.stream(main):
+                    for _ in range(4):
+                        torch.matmul(a, a, out=c)
+                    ev = torch.cuda.Event()
+                    ev.record(main)
+                side.wait_event(ev)
+                s.transfer((l, l + 1), side.cuda_stream)
+            torch.cuda.synchronize()
+            s.status()
+        assert np.array_equal(host(dst_t), want)
+    finally:
+        B.pdkv_tune("max_ctas", 0)
+        if part:
+            torch.cuda.synchronize()
+            del main, side
+            B.pdkv_sm_partition_destroy(part)
+
+
+def test_address_coded_values_name_where_a_row_came_from(oracle):
+    """Every source element carries its own logical coordinate (request, token, layer, K/V,
+    head, dim) as a unique 16-bit code, so a misplaced row would not only differ from the
+    checker: the decoded value says which coordinate landed in its place.  The decode pool is
+    also read back through reshape / index / transpose views (no offset formula) and must
+    list the codes of every request in coordinate order."""
+    from paper_2408_08147_b200.session import TransferSession
+
+    L, H, D = 2, 2, 8
+    lens = np.array([150, 1, 97, 0, 260], np.int32)
+    assert int(lens.sum()) * 2 * L * H * D < 65535
+    w = W.build_workload("coded", 99, num_layers=L, num_kv_heads=H, head_dim=D, elem_bytes=2, seq_len=lens,
+                         src_layout=W.BLOCK_MAJOR, src_block=16, dst_layout=W.LAYER_MAJOR, dst_block=32,
+                         src_slack=1.3, dst_slack=1.3)
+    b = w.batch
+    per_tok = 2 * L * H * D
+    first_tok = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+
+    def decode(code):
+        i = int(code) - 1
+        g, rest = divmod(i, per_tok)
+        r = int(np.searchsorted(first_tok, g, side="right") - 1)
+        l, rest = divmod(rest, 2 * H * D)
+        c, rest = divmod(rest, H * D)
+        h, d = divmod(rest, D)
+        return dict(r=r, t=g - int(first_tok[r]), l=l, c=c, h=h, d=d)
+
+    src6 = np.full(w.src.shape(), SENT, np.uint16)                 # [NB][L][2][B][H][D]
+    Bp = w.src.block_tokens
+    for r in range(b.n_req):
+        for t in range(int(lens[r])):
+            blk = int(b.src_tbl[b.src_tbl_off[r] + t // Bp])
+            base = (int(first_tok[r]) + t) * per_tok + 1
+            src6[blk, :, :, t % Bp] = (base + np.arange(per_tok)).reshape(L, 2, H, D)
+    src = src6.reshape(-1)
+    sent = W.sentinel_pool_numpy(w.dst)
+    want = sent.copy()
+    oracle.transfer(w.src, src, w.dst, want, b)
+    src_t, dst_t = dev(src), dev(sent)
+    torch.cuda.synchronize()
+    with TransferSession(w.src, src_t, w.dst, dst_t, b) as s:
+        buf_t = torch.zeros(s.buffer_bytes, dtype=torch.uint8, device="cuda")
+        s.pack(buf_t)
+        s.status()
+        packed = host(buf_t)
+        s.transfer()
+        s.status()
+    got = host(dst_t)
+    bad = np.flatnonzero(got != want)
+    if bad.size:
+        i = int(bad[0])
+        here = "pad or untouched" if want[i] in (0, SENT) else decode(want[i])
+        there = "zero or sentinel" if got[i] in (0, SENT) else decode(got[i])
+        pytest.fail(f"{bad.size} decode-pool elements differ; element {i} should hold {here} but holds {there}")
+    # the contiguous buffer is the coordinates in order: request, layer, K/V, token, head, dim
+    want_buf = np.concatenate([((int(first_tok[r]) + np.arange(int(lens[r])))[None, None, :, None] * per_tok + 1 +
+                                (np.arange(L)[:, None, None, None] * 2 + np.arange(2)[None, :, None, None]) * H * D +
+                                np.arange(H * D)[None, None, None, :]).reshape(-1) for r in range(b.n_req)])
+    assert np.array_equal(packed, want_buf.astype(np.uint16))
+    # decode pool through views: [L][2][NB][H][B][D] -> per request [L][2][token][H][D]
+    d6 = got.reshape(w.dst.shape())
+    Bd = w.dst.block_tokens
+    for r in range(b.n_req):
+        n = int(lens[r])
+        if n == 0:
+            continue
+        ids = b.dst_tbl[b.dst_tbl_off[r]:b.dst_tbl_off[r] + -(-n // Bd)].astype(np.int64)
+        x = d6[:, :, ids].transpose(0, 1, 2, 4, 3, 5).reshape(L, 2, -1, H, D)       # tokens of the request in order
+        codes = x[:, :, :n].transpose(2, 0, 1, 3, 4).reshape(n, per_tok).astype(np.int64)
+        expect = (int(first_tok[r]) + np.arange(n))[:, None] * per_tok + 1 + np.arange(per_tok)[None, :]
+        assert np.array_equal(codes, expect), f"request {r}: first wrong element holds {decode(codes[codes != expect][0])}"
+        assert (x[:, :, n:] == 0).all()                                             # tail slots of the last block

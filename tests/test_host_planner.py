@@ -445,5 +445,11 @@ def test_chooser_classes_of_copy():
     pack, unpack, fused = shapes(W.make_config(3, n_req=4, head_dim=80))      # 160-byte rows
     assert pack["src_order"] == 0 and unpack["src_order"] == 1 and fused["src_order"] == 1
     assert all(s["vec_bytes"] == 32 for s in (pack, unpack, fused))
+    # 27.5 KiB tiles out of the buffer: staged transpose; 20 KiB tiles out of 16-token blocks: register copy
+    assert (pack["variant"], unpack["variant"], fused["variant"]) == (0, 3, 0)
+    pack, unpack, fused = shapes(W.make_config(4, n_req=2, head_dim=96))      # 192-byte rows, tiles of 24 KiB and more
+    assert (pack["variant"], unpack["variant"], fused["variant"]) == (0, 3, 3)
+    pack, unpack, fused = shapes(W.make_config(4, n_req=2))                   # 256-byte rows: register copy, write order
+    assert (pack["variant"], unpack["variant"], fused["variant"]) == (0, 0, 0) and fused["src_order"] == 0
     pack, unpack, fused = shapes(W.make_config(3, n_req=4, num_kv_heads=1))   # 4 KiB tiles: groups of threads
     assert fused["group_threads"] < fused["threads"] and fused["group_threads"] % 32 == 0
