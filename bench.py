@@ -34,15 +34,15 @@ KERNEL_SOURCE = os.path.join(ROOT, "paper_2408_08147_b200", "csrc", "pdkv_copy_k
 
 # DRAM traffic per launch from ncu (dram__bytes_read.sum + dram__bytes_write.sum),
 # keyed by (workload, op); valid only while the kernel source hashes to KERNEL_SHA.
-# Captured on a 1/8-size case (4 of 32 requests; profiles/copy_tiles_kernel_config2_small_ncu_full.md)
-# and scaled by 8: traffic is proportional to the tokens moved (read 1.0738 GB + write 1.031 GB
-# per 2.1475 GB algorithmic).
-# Config 4 likewise on 2 of 16 requests x 16 of 80 layers (profiles/copy_tiles_kernel_config4_small_ncu_full.md), scaled by 40.
-NCU_TRAFFIC: dict = {(2, "pack"): 8 * (1.074156e9 + 1.028752e9), (2, "unpack"): 8 * (1.073918e9 + 1.030543e9),
-                     (2, "fused"): 8 * (1.074030e9 + 1.029745e9),
-                     (4, "pack"): 40 * (536.931584e6 + 486.842368e6), (4, "unpack"): 40 * (536.926976e6 + 487.005696e6),
-                     (4, "fused"): 40 * (536.943360e6 + 490.336768e6)}
-NCU_KERNEL_SHA = "7e27088e22471cf0"
+# Config 2 was captured on a 1/8-size case (4 of 32 requests; profiles/copy_tiles_kernel_config2_small_ncu_full.md)
+# and is scaled by 8; config 4 on 2 of 16 requests x 16 of 80 layers (profiles/copy_tiles_kernel_config4_small_ncu_full.md),
+# scaled by 40: traffic is proportional to the tokens and layers moved (read = algorithmic to 4 digits, write 4-9% lower
+# because the last dirty lines are still in L2 when the short captured kernel ends).
+NCU_TRAFFIC: dict = {(2, "pack"): 8 * (1.073907e9 + 1.027236e9), (2, "unpack"): 8 * (1.073925e9 + 1.030098e9),
+                     (2, "fused"): 8 * (1.073890e9 + 1.029618e9),
+                     (4, "pack"): 40 * (536.947456e6 + 487.791104e6), (4, "unpack"): 40 * (536.952832e6 + 487.834880e6),
+                     (4, "fused"): 40 * (536.975616e6 + 489.023744e6)}
+NCU_KERNEL_SHA = "d0ad449cc21aa769"
 
 
 def log(*a):

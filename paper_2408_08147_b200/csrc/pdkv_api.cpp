@@ -497,7 +497,10 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
     // that is read is 3-13% faster for every row size except multiples of 256 bytes, where the
     // order of the side that is written wins by 5%.
     out->src_order = o.src_order >= 0 ? o.src_order : ((!flat && row % 256 != 0) ? 1 : 0);
-    cfg.stages = o.stages;
+    // The staged transpose keeps stages x tile bytes of loads in flight per CTA; with two CTAs per SM
+    // two stages are the measured optimum (three: -10% on 32 KiB tiles), so the automatic choice uses
+    // two whatever "stages" says for the bulk-copy variants.
+    cfg.stages = (cfg.variant == 3 && o.variant < 0) ? 2 : o.stages;
     cfg.max_tile_bytes = pl->max_tile_bytes;
 }
 
