@@ -424,7 +424,6 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
         out->lc_skew_shift = (int32_t)shift;
     }
     LaunchConfig &cfg = out->cfg;
-    cfg.group_threads = 0;
     cfg.vec_bytes = pl->vec_bytes;
     if (pl->vec_bytes == 16 && o.vec32 && pl->row_bytes % 32 == 0 &&
         ((reinterpret_cast<uintptr_t>(src.base) | reinterpret_cast<uintptr_t>(dst.base)) & 31u) == 0)
@@ -475,15 +474,17 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
             cfg.unroll = 4;
             cfg.threads = 256;
         }
-        if (cfg.variant == 3 && cfg.threads == 0) {   // staged transpose: 256 threads store what one warp's bulk loads fetched
+        // staged transpose: 256 threads store what one warp's bulk loads fetched (and 256 x 4 is what
+        // the register copy runs if the launch turns out not to qualify for the staged kernel)
+        const bool staged = cfg.variant == 3 && cfg.threads == 0 && cfg.unroll == 0;
+        if (staged) {
             cfg.threads = 256;
             cfg.unroll = 4;
-            if (o.group_threads == 0) cfg.group_threads = 256;
         }
         if (cfg.unroll == 0) cfg.unroll = (flat || small) ? 1 : 4;
         if (cfg.threads == 0) cfg.threads = (flat || small) ? 512 : 256;
-        if (cfg.group_threads == 0 || cfg.variant != 3) cfg.group_threads = o.group_threads;
-        if ((use_tuned || odd_tile) && cfg.group_threads == 0) cfg.group_threads = cfg.threads;
+        cfg.group_threads = o.group_threads;
+        if ((use_tuned || odd_tile || staged) && cfg.group_threads == 0) cfg.group_threads = cfg.threads;
         if (cfg.group_threads == 0) {
             const int64_t vecs = std::max<int64_t>(1, pl->mean_tile_bytes[op] / cfg.vec_bytes);
             const int64_t want = vecs / ((flat || small) ? 2 : cfg.unroll);

@@ -240,3 +240,8 @@ def test_config3_full_size_rows_of_160_bytes(oracle):
 
 def test_config5_full_size_rows_of_160_bytes(oracle):
     run_fullsize(oracle, W.make_config(5, head_dim=80), n_sample=0, seed=35, group=16)
+
+
+def test_config4_full_size_rows_of_192_bytes(oracle):
+    """70B-shaped with head_dim 96: unpack and fused both run the staged transpose (tiles of 32 KiB)."""
+    run_fullsize(oracle, W.make_config(4, head_dim=96), n_sample=0, seed=36, group=2)
