@@ -773,7 +773,8 @@ def overlap_arm(args):
                       {"variant": 0, "ctas_per_sm": 2}, sms))
     defaults = {k: B.pdkv_tune_get(k) for k in ("variant", "ctas_per_sm", "threads", "unroll", "tile_bytes", "stages",
                                                 "max_ctas", "group_threads")}
-    t_compute, _ = timed(compute_on(plain_main), args.steps, plain_main, plain_side)
+    with ClockSampler(0) as clk0:
+        t_compute, _ = timed(compute_on(plain_main), args.steps, plain_main, plain_side)
     results = {}
     for name, tune, special in modes:
         main, side, part = plain_main, plain_side, None
@@ -811,7 +812,9 @@ def overlap_arm(args):
 
         t_c, _ = timed(compute_on(main), args.steps, main, side) if part else (t_compute, None)
         t_x, _ = timed(transfer_only, args.steps, main, side)
-        t_o, t_o_main = timed(overlapped, args.steps, main, side)
+        with ClockSampler(0) as clk:
+            t_o, t_o_main = timed(overlapped, args.steps, main, side)
+        rec["clocks_while_overlapped"] = clk.summary()
         rec.update({"compute_alone_ms": t_c, "transfer_alone_ms": t_x, "overlapped_ms": t_o,
                     "compute_sequence_while_overlapped_ms": t_o_main,
                     "serial_ms": t_c + t_x,
@@ -838,7 +841,7 @@ def overlap_arm(args):
     out = {"mode": "overlap", "config": {"workload": workload_name(w), "layers": L,
                                          "compute_stand_in": f"{L} x torch.matmul bf16 {n}^3 on the main stream",
                                          "transfer_stream_priority": "high" if args.side_priority else "default"},
-           "compute_alone_ms": t_compute, "variants": results}
+           "compute_alone_ms": t_compute, "clocks_compute_alone": clk0.summary(), "variants": results}
     print(json.dumps(out), flush=True)
 
 
