@@ -175,7 +175,9 @@ int pdkv_plan_destroy(pdkv_plan *plan);
  * if `buf` is given: device, at least pdkv_plan_buffer() bytes) and for
  * transfer; a shape replaces the built-in one only if it is more than 2.5%
  * faster.  With a block-major pool the strip skew (see "lc_skew") is also timed
- * the other way round than its stride rule decides, and kept on the same terms.  The operations are the real ones: afterwards `buf` holds the packed
+ * the other way round than its stride rule decides, and kept on the same terms;
+ * so is the other kernel for tiles that are transposed on the way (register copy
+ * against staged transpose, see "variant"; pdkv_plan_launch_shape() shows the outcome).  The operations are the real ones: afterwards `buf` holds the packed
  * layers and the decode pool the transferred layers that were used for timing
  * (with an unpack-only plan `buf` must already hold a packed batch).  The
  * call synchronises `stream` repeatedly; it is meant for set-up time, once per
