@@ -55,6 +55,17 @@ int main(void)
            (long long)tiles[0].src_off, (long long)tiles[0].dst_off, (int)tiles[0].ntok);
     if ((rc = pdkv_plan_launches(plan, PDKV_OP_PACK, &launches)) != PDKV_OK) return 34;
     printf("pack_launches %lld\n", (long long)launches);
+    {   /* what the plan would launch, and that it keeps the tunables it was created with */
+        pdkv_launch_shape shape;
+        int64_t frozen = -1;
+        if ((rc = pdkv_plan_launch_shape(plan, PDKV_OP_TRANSFER, 0, 2, &shape)) != PDKV_OK) return 35;
+        if ((rc = pdkv_tune("ctas_per_sm", 7)) != PDKV_OK) return 36;
+        if ((rc = pdkv_plan_option(plan, "ctas_per_sm", &frozen)) != PDKV_OK) return 37;
+        if ((rc = pdkv_tune("ctas_per_sm", 2)) != PDKV_OK) return 38;
+        printf("launch_shape %d %d %d %d %lld\n", (int)shape.threads, (int)shape.vec_bytes, (int)shape.ctas_per_sm,
+               (int)shape.variant, (long long)frozen);
+        if (pdkv_plan_launch_shape(plan, PDKV_OP_TRANSFER, 1, 3, &shape) != PDKV_ERR_INVALID_ARG) return 39;
+    }
     /* a dry-run plan cannot be launched */
     printf("transfer_on_dry_plan %d\n", pdkv_transfer(plan, 0, 2, NULL));
 
