@@ -786,7 +786,6 @@ def overlap_arm(args):
                 got_t, got_c = B.pdkv_sm_partition_info(part)
                 side = torch.cuda.ExternalStream(B.pdkv_sm_partition_stream(part, 0))
                 main = torch.cuda.ExternalStream(B.pdkv_sm_partition_stream(part, 1))
-                tune["max_ctas"] = got_t * tune["ctas_per_sm"]
                 rec["sm_partition"] = {"transfer_sms": got_t, "compute_sms": got_c}
         except B.PdkvError as e:
             results[name] = {"unavailable": str(e)}

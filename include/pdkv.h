@@ -362,8 +362,8 @@ int pdkv_queue_destroy(pdkv_queue *queue);
  * non-blocking stream: kernels enqueued on stream 0 (`which` = 0) run only on the
  * transfer SMs, kernels on stream 1 only on the others, so neither waits for a CTA
  * slot of the other.  Streams belong to the partition; use them like any
- * cudaStream_t (for pdkv_transfer create the plan with "max_ctas" =
- * transfer SMs x "ctas_per_sm", so that the persistent grid matches its share).
+ * cudaStream_t.  A pack / unpack / transfer call given a partition's stream sizes
+ * its persistent grid to that partition's SMs ("ctas_per_sm" CTAs on each) by itself.
  * Nothing outlasts the process and no device setting changes.  (No counterpart in
  * the paper, whose transfer engine is not the compute device.)
  * Errors: INVALID_ARG, NOMEM, CUDA (driver without green contexts, or a split the

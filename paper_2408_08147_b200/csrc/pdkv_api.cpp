@@ -266,7 +266,8 @@ int launch_op(const pdkv_plan *pl, int op, const pdkv::Side &src, const pdkv::Si
     p.H = pl->H;
     p.row_bytes = (int32_t)pl->row_bytes;
     pdkv::ResolvedLaunch r;
-    pdkv::resolve_launch(pl, op, src, dst, p.n_lc, pl->sm_count, &r);
+    const int share = pdkv::partition_sms_of(stream);   // a stream of an SM partition: the grid fits its share
+    pdkv::resolve_launch(pl, op, src, dst, p.n_lc, share > 0 ? share : pl->sm_count, &r);
     p.lc_fastest = r.lc_fastest;
     p.chunked = r.chunked;
     p.lc_skew = r.lc_skew;

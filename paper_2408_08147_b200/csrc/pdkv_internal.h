@@ -145,6 +145,9 @@ void resolve_launch(const pdkv_plan *plan, int op, const Side &src, const Side &
 void describe_transfer(const pdkv_plan *plan, Side *src, Side *dst, int *H, int *row_bytes,
                        int *vec_bytes, int *num_layers, int *device);
 int report_cuda_error(cudaError_t e, const char *what);
+// SMs of the partition a stream belongs to (a stream handed out by pdkv_sm_partition_stream), else 0:
+// launches on such a stream size their persistent grid to the partition's share.
+int partition_sms_of(cudaStream_t stream);
 int plan_num_layers(const pdkv_plan *plan);
 
 }  // namespace pdkv

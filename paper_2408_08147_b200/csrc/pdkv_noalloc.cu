@@ -109,7 +109,8 @@ extern "C" int pdkv_transfer_noalloc(const pdkv_pool *src, const pdkv_pool *dst,
         p.row_bytes = row_bytes;
         // launch shape, work order and strip skew from the chooser every plan-based call uses
         pdkv::ResolvedLaunch r;
-        pdkv::resolve_launch(plan.p, PDKV_OP_TRANSFER, p.src, p.dst, p.n_lc, slot.sm_count, &r);
+        const int share = pdkv::partition_sms_of(st);
+        pdkv::resolve_launch(plan.p, PDKV_OP_TRANSFER, p.src, p.dst, p.n_lc, share > 0 ? share : slot.sm_count, &r);
         p.lc_fastest = r.lc_fastest;
         p.chunked = r.chunked;
         p.lc_skew = r.lc_skew;

@@ -7,8 +7,11 @@
 // an object of this process's primary context and dies with it.
 //
 // The driver entry points are looked up at run time (the library links only the runtime).
+#include <atomic>
 #include <mutex>
 #include <new>
+#include <utility>
+#include <vector>
 
 #include <cuda.h>
 
@@ -53,7 +56,43 @@ const Driver &driver()
     return d;
 }
 
+// Streams of live partitions with their SM counts, so that a launch can size its grid to the
+// share of the stream it is given.  Read on every launch: the count keeps the common case
+// (no partition exists) to one relaxed load.
+std::mutex g_streams_mutex;
+std::vector<std::pair<cudaStream_t, int>> g_streams;
+std::atomic<int> g_stream_count{0};
+
+void register_stream(cudaStream_t st, int sms)
+{
+    std::lock_guard<std::mutex> lock(g_streams_mutex);
+    g_streams.emplace_back(st, sms);
+    g_stream_count.store((int)g_streams.size(), std::memory_order_release);
+}
+
+void unregister_stream(cudaStream_t st)
+{
+    std::lock_guard<std::mutex> lock(g_streams_mutex);
+    for (size_t i = 0; i < g_streams.size(); ++i)
+        if (g_streams[i].first == st) {
+            g_streams.erase(g_streams.begin() + (long)i);
+            break;
+        }
+    g_stream_count.store((int)g_streams.size(), std::memory_order_release);
+}
+
 }  // namespace
+
+namespace pdkv {
+int partition_sms_of(cudaStream_t stream)
+{
+    if (g_stream_count.load(std::memory_order_acquire) == 0) return 0;
+    std::lock_guard<std::mutex> lock(g_streams_mutex);
+    for (const auto &e : g_streams)
+        if (e.first == stream) return e.second;
+    return 0;
+}
+}  // namespace pdkv
 
 struct pdkv_sm_partition {
     int device = 0;
@@ -98,6 +137,7 @@ int pdkv_sm_partition_create(int device, int transfer_sms, pdkv_sm_partition **o
         if (d.GreenCtxStreamCreate(&p->stream[i], p->ctx[i], CU_STREAM_NON_BLOCKING, 0) != CUDA_SUCCESS)
             return fail("cuGreenCtxStreamCreate");
         p->sms[i] = (int)res[i]->sm.smCount;
+        register_stream(p->stream[i], p->sms[i]);
     }
     *out = p;
     return PDKV_OK;
@@ -125,6 +165,7 @@ int pdkv_sm_partition_destroy(pdkv_sm_partition *p)
     pdkv::DeviceGuard guard(p->device);
     for (int i = 0; i < 2; ++i) {
         if (p->stream[i]) {
+            unregister_stream(p->stream[i]);
             cudaStreamSynchronize(p->stream[i]);
             d.StreamDestroy(p->stream[i]);
         }
