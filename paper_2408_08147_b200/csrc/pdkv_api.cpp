@@ -386,8 +386,44 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
                     ResolvedLaunch *out)
 {
     const LaunchOptions &o = pl->opt;
+    LaunchConfig &cfg = out->cfg;
+    const int64_t hrow = pl->hrow_bytes, row = pl->row_bytes;
+    const bool flat = src.head_stride == row && src.tok_stride == hrow && dst.head_stride == row &&
+                      dst.tok_stride == hrow;
+    const bool small = pl->mean_tile_bytes[op] < 24 * 1024;
     out->lc_fastest = o.lc_fastest;
     out->chunked = o.chunked;
+    bool strip_first_rule = false;
+    {   // Kernel.  Automatic: the register copy, except for tiles that go from a token-major side to
+        // a head-major one in rows of more than 128 bytes that are not multiples of 256 (head sizes
+        // such as 80, 96 or 112 at 2 bytes).  Those run the staged transpose, whose reads and writes
+        // are both contiguous runs: measured on 8B- and 70B-shaped batches with 80 to 192 dims per
+        // head, +3 to +12% over the register copy for tiles of 24 KiB and more.  Smaller tiles of such
+        // rows (16 to 24 KiB: 16-token prefill blocks) gain 5-9% from it only in the fused call out of
+        // a block-major pool and only with the work order turned round -- consecutive CTAs take the
+        // consecutive (layer, K/V) strips of one block, which are one contiguous stretch of the pool --
+        // and three stages; every other combination (256- and 128-byte rows, other calls) is slower
+        // that way.  pdkv_plan_autotune() may have timed the other kernel.
+        int variant = o.variant;
+        if (variant < 0) {
+            const bool tok_to_head = src.tok_stride >= src.head_stride && dst.tok_stride < dst.head_stride;
+            const bool odd_rows = row % 256 != 0 && row > 128 && row % 16 == 0;
+            variant = 0;
+            if (tok_to_head && odd_rows && !small) {
+                variant = 3;
+            } else if (tok_to_head && odd_rows && op == PDKV_OP_TRANSFER && pl->mean_tile_bytes[op] >= 16 * 1024 &&
+                       pl->src.d.layout == PDKV_LAYOUT_BLOCK_MAJOR && o.lc_fastest == 0 && n_lc >= 16) {
+                variant = 3;
+                strip_first_rule = true;
+            }
+            if (pl->shape[op].variant >= 0) {
+                variant = pl->shape[op].variant;
+                strip_first_rule = strip_first_rule && variant == 3;
+            }
+        }
+        cfg.variant = variant;
+        if (strip_first_rule) out->lc_fastest = 1;
+    }
     {   // Strip skew (see pdkv_tune "lc_skew").  Automatic: only for calls that read (or, failing
         // that, write) a block-major pool whose block stride, stripped of its factors of two, is
         // divisible by 3, 5 or 17 (e.g. 80 layers x 64 tokens x 2 KiB = 5 x 4 MiB).  With such
@@ -424,7 +460,6 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
         out->lc_skew = out->lc_fastest ? 0 : (int32_t)skew;
         out->lc_skew_shift = (int32_t)shift;
     }
-    LaunchConfig &cfg = out->cfg;
     cfg.vec_bytes = pl->vec_bytes;
     if (pl->vec_bytes == 16 && o.vec32 && pl->row_bytes % 32 == 0 &&
         ((reinterpret_cast<uintptr_t>(src.base) | reinterpret_cast<uintptr_t>(dst.base)) & 31u) == 0)
@@ -436,24 +471,6 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
     cfg.sm_count = sm_count;
     cfg.elem_bytes = pl->E;
     cfg.check_bounds = o.debug_bounds != 0;
-    const int64_t hrow = pl->hrow_bytes, row = pl->row_bytes;
-    const bool flat = src.head_stride == row && src.tok_stride == hrow && dst.head_stride == row &&
-                      dst.tok_stride == hrow;
-    const bool small = pl->mean_tile_bytes[op] < 24 * 1024;
-    {   // Kernel.  Automatic: the register copy, except for tiles that go from a token-major side to
-        // a head-major one in rows of more than 128 bytes that are not multiples of 256 (head sizes
-        // such as 80, 96 or 112 at 2 bytes): those run the staged transpose, whose reads and writes are both contiguous runs
-        // (measured on 8B- and 70B-shaped batches with 80 to 192 dims per head: +3 to +12% over the
-        // register copy for tiles of 24 KiB and more; for smaller tiles and for 256-byte rows the
-        // register copy stays ahead).  pdkv_plan_autotune() may have timed the other choice.
-        int variant = o.variant;
-        if (variant < 0) {
-            const bool tok_to_head = src.tok_stride >= src.head_stride && dst.tok_stride < dst.head_stride;
-            variant = (tok_to_head && row % 256 != 0 && row > 128 && row % 16 == 0 && !small) ? 3 : 0;
-            if (pl->shape[op].variant >= 0) variant = pl->shape[op].variant;
-        }
-        cfg.variant = variant;
-    }
     {   // Automatic launch shape, measured best per class of copy on B200.  Full tiles
         // (about 32 KiB): a flat copy (token-major on both sides) runs 512 threads with
         // one access in flight each, i.e. two passes per tile; a copy with a head-major
@@ -501,8 +518,8 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
     out->src_order = o.src_order >= 0 ? o.src_order : ((!flat && row % 256 != 0) ? 1 : 0);
     // The staged transpose keeps stages x tile bytes of loads in flight per CTA; with two CTAs per SM
     // two stages are the measured optimum (three: -10% on 32 KiB tiles), so the automatic choice uses
-    // two whatever "stages" says for the bulk-copy variants.
-    cfg.stages = (cfg.variant == 3 && o.variant < 0) ? 2 : o.stages;
+    // two whatever "stages" says for the bulk-copy variants (three for the strip-first order of 16-24 KiB tiles).
+    cfg.stages = (cfg.variant == 3 && o.variant < 0) ? (strip_first_rule ? 3 : 2) : o.stages;
     cfg.max_tile_bytes = pl->max_tile_bytes;
 }
 
@@ -853,9 +870,13 @@ int pdkv_plan_autotune(pdkv_plan *plan, void *buf, size_t buf_bytes, void *strea
         if (rc == PDKV_OK && plan->opt.variant < 0 && op != PDKV_OP_PACK && plan->has_dst &&
             plan->dst.d.layout == PDKV_LAYOUT_LAYER_MAJOR && (op == PDKV_OP_UNPACK || plan->src.d.layout == PDKV_LAYOUT_BLOCK_MAJOR) &&
             plan->row_bytes % 16 == 0) {
-            const bool rule_staged = plan->row_bytes % 256 != 0 && plan->row_bytes > 128 && plan->mean_tile_bytes[op] >= 24 * 1024;
+            const pdkv::Side buf_side = buffer_side(nullptr, 0, plan->row_bytes, plan->hrow_bytes);
+            pdkv::ResolvedLaunch by_rule;
+            plan->shape[op] = pdkv_plan::Shape();
+            pdkv::resolve_launch(plan, op, op == PDKV_OP_UNPACK ? buf_side : pool_side(plan->src, plan->row_bytes, plan->hrow_bytes),
+                                 pool_side(plan->dst, plan->row_bytes, plan->hrow_bytes), 2 * layers, plan->sm_count, &by_rule);
             pdkv_plan::Shape other;
-            other.variant = rule_staged ? 0 : 3;
+            other.variant = by_rule.cfg.variant == 3 ? 0 : 3;
             plan->shape[op] = other;
             float ms = 0.f;
             rc = time_ms(op, &ms);

@@ -445,8 +445,10 @@ def test_chooser_classes_of_copy():
     pack, unpack, fused = shapes(W.make_config(3, n_req=4, head_dim=80))      # 160-byte rows
     assert pack["src_order"] == 0 and unpack["src_order"] == 1 and fused["src_order"] == 1
     assert all(s["vec_bytes"] == 32 for s in (pack, unpack, fused))
-    # 27.5 KiB tiles out of the buffer: staged transpose; 20 KiB tiles out of 16-token blocks: register copy
-    assert (pack["variant"], unpack["variant"], fused["variant"]) == (0, 3, 0)
+    # 27.5 KiB tiles out of the buffer: staged transpose; 20 KiB tiles out of 16-token blocks: staged transpose
+    # with the strips of one block on consecutive CTAs (and therefore no strip skew)
+    assert (pack["variant"], unpack["variant"], fused["variant"]) == (0, 3, 3)
+    assert (unpack["lc_fastest"], fused["lc_fastest"], fused["lc_skew"]) == (0, 1, 0)
     pack, unpack, fused = shapes(W.make_config(4, n_req=2, head_dim=96))      # 192-byte rows, tiles of 24 KiB and more
     assert (pack["variant"], unpack["variant"], fused["variant"]) == (0, 3, 3)
     pack, unpack, fused = shapes(W.make_config(4, n_req=2))                   # 256-byte rows: register copy, write order
