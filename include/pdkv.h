@@ -416,7 +416,8 @@ int pdkv_plan_option(const pdkv_plan *plan, const char *key, int64_t *value);
  * copies them into the plan (pdkv_transfer_noalloc() reads them at the call); changing
  * them never affects a plan that already exists.
  *   "tile_bytes"     target bytes moved per tile (default 32768)
- *   "ctas_per_sm"    persistent CTAs per SM (default 2)
+ *   "ctas_per_sm"    persistent CTAs per SM; 0 (default) = automatic: 2, or 3 for row-permuting
+ *                    copies of 12-16 KiB tiles (which then run 256 threads x 2 accesses)
  *   "max_ctas"       cap on the grid size, 0 = none (default).  A small grid
  *                    leaves most SMs to other kernels of the process at a
  *                    proportionally lower copy rate

@@ -499,10 +499,22 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
             cfg.threads = 256;
             cfg.unroll = 4;
         }
+        // Row-permuting copies of 12-16 KiB tiles (16-token blocks of 128-byte rows: 1-byte elements or
+        // 64 dims per head; four KV heads; 8-token blocks): one pass of 256 threads x 2 accesses per tile
+        // and three CTAs per SM, i.e. 48 KiB in flight per SM.  Measured on six such batches: +7 to +16%
+        // over two passes of 512 x 1 (5.5-5.9 -> 6.2-6.6 TB/s); tiles of 8 KiB and of 32 KiB lose with it.
+        const int64_t mean_vecs = pl->mean_tile_bytes[op] / cfg.vec_bytes;
+        const bool half_tile = !flat && !use_tuned && !odd_tile && cfg.variant == 0 && cfg.threads == 0 && cfg.unroll == 0 &&
+                               o.group_threads == 0 && mean_vecs > 384 && mean_vecs <= 576;   // (zero-fill tiles may be larger)
+        if (half_tile) {
+            cfg.threads = 256;
+            cfg.unroll = 2;
+            if (cfg.ctas_per_sm == 0) cfg.ctas_per_sm = 3;
+        }
         if (cfg.unroll == 0) cfg.unroll = (flat || small) ? 1 : 4;
         if (cfg.threads == 0) cfg.threads = (flat || small) ? 512 : 256;
         cfg.group_threads = o.group_threads;
-        if ((use_tuned || odd_tile || staged) && cfg.group_threads == 0) cfg.group_threads = cfg.threads;
+        if ((use_tuned || odd_tile || staged || half_tile) && cfg.group_threads == 0) cfg.group_threads = cfg.threads;
         if (cfg.group_threads == 0) {
             const int64_t vecs = std::max<int64_t>(1, pl->mean_tile_bytes[op] / cfg.vec_bytes);
             const int64_t want = vecs / ((flat || small) ? 2 : cfg.unroll);
@@ -510,12 +522,14 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
             while (g < want && g < cfg.threads) g *= 2;
             cfg.group_threads = g;
         }
+        if (cfg.ctas_per_sm == 0) cfg.ctas_per_sm = 2;
     }
     // Row order inside a tile of the register copy (see CopyParams::src_order).  Measured on
     // transposing copies with rows of 128 to 384 bytes: walking the rows in the order of the side
-    // that is read is 3-13% faster for every row size except multiples of 256 bytes, where the
-    // order of the side that is written wins by 5%.
-    out->src_order = o.src_order >= 0 ? o.src_order : ((!flat && row % 256 != 0) ? 1 : 0);
+    // that is read is 3-13% faster for rows of more than 128 bytes that are not multiples of 256, and
+    // for 128-byte rows in tiles under 24 KiB; for multiples of 256 bytes, and for 128-byte rows in
+    // full tiles, the order of the side that is written wins by 5-10%.
+    out->src_order = o.src_order >= 0 ? o.src_order : ((!flat && row % 256 != 0 && (row > 128 || small)) ? 1 : 0);
     // The staged transpose keeps stages x tile bytes of loads in flight per CTA; with two CTAs per SM
     // two stages are the measured optimum (three: -10% on 32 KiB tiles), so the automatic choice uses
     // two whatever "stages" says for the bulk-copy variants (three for the strip-first order of 16-24 KiB tiles).
@@ -851,6 +865,7 @@ int pdkv_plan_autotune(pdkv_plan *plan, void *buf, size_t buf_bytes, void *strea
         add(256, 4, 2); add(512, 1, 2); add(512, 2, 2); add(256, 1, 4); add(1024, 1, 1); add(256, 2, 2);
         add(nvec, 1, 2); add((nvec + 1) / 2, 2, 2); add((nvec + 3) / 4, 4, 2);       // one pass = one tile
         add((nvec + 1) / 2, 1, 2); add((nvec + 3) / 4, 2, 2);                         // two passes = one tile
+        add((nvec + 1) / 2, 2, 3); add((nvec + 3) / 4, 4, 3); add((nvec + 3) / 4, 4, 4);   // one pass, more CTAs per SM
         plan->shape[op] = pdkv_plan::Shape();
         float best_ms = 0.f;
         rc = time_ms(op, &best_ms);              // the per-class default is the incumbent
@@ -1244,7 +1259,7 @@ int pdkv_tune(const char *key, int64_t value)
     pdkv::Tunables &t = pdkv::tunables();
     const std::string k(key);
     if (k == "tile_bytes" && value >= 1 && value <= (1ll << 30)) t.tile_bytes = value;
-    else if (k == "ctas_per_sm" && value >= 1 && value <= 32) t.ctas_per_sm = value;
+    else if (k == "ctas_per_sm" && value >= 0 && value <= 32) t.ctas_per_sm = value;
     else if (k == "max_ctas" && value >= 0 && value <= 65535) t.max_ctas = value;
     else if (k == "threads" && (value == 0 || (value >= 32 && value <= 1024 && value % 32 == 0))) t.threads = value;
     else if (k == "unroll" && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8)) t.unroll = value;

@@ -96,7 +96,7 @@ struct DeviceGuard {
 // Process-wide settings; atomics because pdkv_tune may race with launches on other threads.
 struct Tunables {
     std::atomic<int64_t> tile_bytes{32768};
-    std::atomic<int64_t> ctas_per_sm{2};
+    std::atomic<int64_t> ctas_per_sm{0};   // 0: chosen per class of copy (2, or 3 for half-size tiles)
     std::atomic<int64_t> max_ctas{0};
     std::atomic<int64_t> threads{0};   // 0: chosen with unroll, per class of copy
     std::atomic<int64_t> unroll{0};    // 0: chosen per class of copy
@@ -120,7 +120,7 @@ Tunables &tunables();
 // launching the way it was set up, whatever pdkv_tune() is told afterwards (by this or
 // another thread).  pdkv_tune() only sets the defaults of plans created later.
 struct LaunchOptions {
-    int ctas_per_sm = 2, max_ctas = 0, threads = 0, unroll = 0, vec32 = 1, lc_fastest = 0, group_threads = 0,
+    int ctas_per_sm = 0, max_ctas = 0, threads = 0, unroll = 0, vec32 = 1, lc_fastest = 0, group_threads = 0,
         chunked = 0, lc_skew = -1, lc_skew_shift = 0, debug_bounds = 0, variant = -1, stages = 3, src_order = -1;
     int64_t debug_shrink = 0;
     int64_t tile_bytes = 32768;

@@ -61,7 +61,7 @@ int main(void)
         if ((rc = pdkv_plan_launch_shape(plan, PDKV_OP_TRANSFER, 0, 2, &shape)) != PDKV_OK) return 35;
         if ((rc = pdkv_tune("ctas_per_sm", 7)) != PDKV_OK) return 36;
         if ((rc = pdkv_plan_option(plan, "ctas_per_sm", &frozen)) != PDKV_OK) return 37;
-        if ((rc = pdkv_tune("ctas_per_sm", 2)) != PDKV_OK) return 38;
+        if ((rc = pdkv_tune("ctas_per_sm", 0)) != PDKV_OK) return 38;
         printf("launch_shape %d %d %d %d %lld\n", (int)shape.threads, (int)shape.vec_bytes, (int)shape.ctas_per_sm,
                (int)shape.variant, (long long)frozen);
         if (pdkv_plan_launch_shape(plan, PDKV_OP_TRANSFER, 1, 3, &shape) != PDKV_ERR_INVALID_ARG) return 39;

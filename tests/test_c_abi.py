@@ -41,7 +41,7 @@ def test_header_is_plain_c_and_callable_from_c(tmp_path):
     assert int(f[2]) == 3 * (2 * 2 * 4 * 2 * 16 * 2) and int(f[4]) == 0 and int(f[6]) == 4
     assert int(got["pack_launches"]) == 1
     # 32-byte rows, tiny tiles: groups of threads in a 512-thread CTA, 32-byte accesses, register copy;
-    # the plan kept "ctas_per_sm" = 2 although the tunable was 7 when it was asked
-    assert [int(x) for x in got["launch_shape"].split()] == [512, 32, 2, 0, 2]
+    # the plan kept "ctas_per_sm" = 0 (automatic: 2 here) although the tunable was 7 when it was asked
+    assert [int(x) for x in got["launch_shape"].split()] == [512, 32, 2, 0, 0]
     assert int(got["transfer_on_dry_plan"]) == -1          # PDKV_ERR_INVALID_ARG
     assert int(got["duplicate_decode_block"]) == -3        # PDKV_ERR_TABLE
