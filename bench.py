@@ -540,7 +540,7 @@ def main_arm(args):
                       "step": "pdkv_pack + pdkv_unpack + pdkv_transfer, all layers",
                       "payload_bytes": sess.buffer_bytes, "step_bytes": step_bytes,
                       "plan_create_destroy_ms": statistics.median(plan_ms),
-                      "autotuned_shapes (threads, unroll, CTAs/SM, strip skew per op; zeros = built-in, skew -1 = stride rule)": tuned,
+                      "autotuned_shapes": tuned,   # (threads, unroll, CTAs/SM, strip skew) per op; zeros = built-in, skew -1 = stride rule
                       "l2": "inputs exceed L2 (pools and buffer are GiB-sized; no flush needed)"
                       if sess.buffer_bytes > (1 << 29) else "L2-resident workload: not an HBM number",
                       "tunables": {k: B.pdkv_tune_get(k) for k in
