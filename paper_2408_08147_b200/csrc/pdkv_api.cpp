@@ -118,6 +118,7 @@ pdkv::Side pool_side(const pdkv_pool &p, int64_t row, int64_t hrow)
         s.tok_stride = row;
         s.head_stride = (int64_t)p.d.block_tokens * row;
     }
+    if (p.d.num_kv_heads == 1) s.head_stride = row;   // one head: the head stride is never applied, and both layouts are token-major
     return s;
 }
 
@@ -461,9 +462,14 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
         out->lc_skew_shift = (int32_t)shift;
     }
     cfg.vec_bytes = pl->vec_bytes;
-    if (pl->vec_bytes == 16 && o.vec32 && pl->row_bytes % 32 == 0 &&
-        ((reinterpret_cast<uintptr_t>(src.base) | reinterpret_cast<uintptr_t>(dst.base)) & 31u) == 0)
-        cfg.vec_bytes = 32;
+    const bool bases32 = ((reinterpret_cast<uintptr_t>(src.base) | reinterpret_cast<uintptr_t>(dst.base)) & 31u) == 0;
+    if (pl->vec_bytes == 16 && o.vec32 && pl->row_bytes % 32 == 0 && bases32) cfg.vec_bytes = 32;
+    if (flat) {   // a flat tile is one run of bytes on both sides, and every tile starts at a multiple of a token's
+                  // bytes: the access width follows from those, whatever the row size (144-byte rows: 32, not 16)
+        int w = (o.vec32 && bases32) ? 32 : 16;
+        while (hrow % w) w >>= 1;
+        if (w > cfg.vec_bytes) cfg.vec_bytes = w;
+    }
     cfg.unroll = o.unroll;
     cfg.threads = o.threads;
     cfg.ctas_per_sm = o.ctas_per_sm;
