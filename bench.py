@@ -38,11 +38,11 @@ KERNEL_SOURCE = os.path.join(ROOT, "paper_2408_08147_b200", "csrc", "pdkv_copy_k
 # and is scaled by 8; config 4 on 2 of 16 requests x 16 of 80 layers (profiles/copy_tiles_kernel_config4_small_ncu_full.md),
 # scaled by 40: traffic is proportional to the tokens and layers moved (read = algorithmic to 4 digits, write 4-9% lower
 # because the last dirty lines are still in L2 when the short captured kernel ends).
-NCU_TRAFFIC: dict = {(2, "pack"): 8 * (1.073860e9 + 1.026701e9), (2, "unpack"): 8 * (1.073865e9 + 1.029703e9),
-                     (2, "fused"): 8 * (1.073890e9 + 1.029696e9),
-                     (4, "pack"): 40 * (536.928256e6 + 487.782912e6), (4, "unpack"): 40 * (536.917760e6 + 490.807552e6),
-                     (4, "fused"): 40 * (536.915456e6 + 488.461568e6)}
-NCU_KERNEL_SHA = "359f82fc577e38b6"
+NCU_TRAFFIC: dict = {(2, "pack"): 8 * (1.073972e9 + 1.027700e9), (2, "unpack"): 8 * (1.073934e9 + 1.030297e9),
+                     (2, "fused"): 8 * (1.073925e9 + 1.030007e9),
+                     (4, "pack"): 40 * (536.960000e6 + 488.121856e6), (4, "unpack"): 40 * (536.996352e6 + 488.964864e6),
+                     (4, "fused"): 40 * (536.962816e6 + 487.982848e6)}
+NCU_KERNEL_SHA = "5333b1c77fb50ab9"
 
 
 def log(*a):

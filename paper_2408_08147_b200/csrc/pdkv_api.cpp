@@ -408,7 +408,9 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
         int variant = o.variant;
         if (variant < 0) {
             const bool tok_to_head = src.tok_stride >= src.head_stride && dst.tok_stride < dst.head_stride;
-            const bool odd_rows = row % 256 != 0 && row > 128 && row % 16 == 0;
+            // (rows under 128 bytes that are not multiples of 64 -- 80, 96 or 112 one-byte elements -- are worse
+            // still on the register copy, 4.4-5.2 TB/s, and reach 5.9-6.4 staged; 64- and 128-byte rows do not)
+            const bool odd_rows = row % 16 == 0 && ((row > 128 && row % 256 != 0) || (row < 128 && row % 64 != 0));
             variant = 0;
             if (tok_to_head && odd_rows && !small) {
                 variant = 3;
@@ -490,10 +492,24 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
             cfg.unroll = tuned.unroll;
             cfg.ctas_per_sm = tuned.ctas_per_sm;
         }
+        // Copies of 9-17 KiB tiles (16-token blocks of 128-byte rows: 1-byte elements or 64 dims per
+        // head; four KV heads; 8-token blocks): one pass of 256 threads x 2 accesses per tile and three
+        // CTAs per SM, i.e. 48 KiB in flight per SM.  Measured on six such batches of row-permuting
+        // copies: +7 to +16% over two passes of 512 x 1 (5.5-5.9 -> 6.2-6.6 TB/s); tiles of 8 KiB, of
+        // 18 KiB and of 32 KiB lose with it.  Flat copies neither gain nor lose at 16 KiB and gain 20%
+        // at 10-14 KiB, so they take it too.  Keyed on this operation's own mean tile.
+        const int64_t mean_vecs = pl->mean_tile_bytes[op] / cfg.vec_bytes;
+        const bool half_tile = !use_tuned && cfg.variant == 0 && cfg.threads == 0 && cfg.unroll == 0 &&
+                               o.group_threads == 0 && mean_vecs > 288 && mean_vecs <= 544;   // (zero-fill tiles may be larger)
+        if (half_tile) {
+            cfg.threads = 256;
+            cfg.unroll = 2;
+            if (cfg.ctas_per_sm == 0) cfg.ctas_per_sm = 3;
+        }
         // Tiles of more than half but less than a full 256 x 4 pass (head sizes, head counts or
         // block sizes that are not powers of two): that one pass, whatever the class of copy.
         const int64_t max_vecs = pl->max_tile_bytes / cfg.vec_bytes;
-        const bool odd_tile = !use_tuned && cfg.unroll == 0 && cfg.threads == 0 && max_vecs > 512 && max_vecs < 1024;
+        const bool odd_tile = !use_tuned && !half_tile && cfg.unroll == 0 && cfg.threads == 0 && max_vecs > 512 && max_vecs < 1024;
         if (odd_tile) {
             cfg.unroll = 4;
             cfg.threads = 256;
@@ -504,18 +520,6 @@ void resolve_launch(const pdkv_plan *pl, int op, const Side &src, const Side &ds
         if (staged) {
             cfg.threads = 256;
             cfg.unroll = 4;
-        }
-        // Row-permuting copies of 12-16 KiB tiles (16-token blocks of 128-byte rows: 1-byte elements or
-        // 64 dims per head; four KV heads; 8-token blocks): one pass of 256 threads x 2 accesses per tile
-        // and three CTAs per SM, i.e. 48 KiB in flight per SM.  Measured on six such batches: +7 to +16%
-        // over two passes of 512 x 1 (5.5-5.9 -> 6.2-6.6 TB/s); tiles of 8 KiB and of 32 KiB lose with it.
-        const int64_t mean_vecs = pl->mean_tile_bytes[op] / cfg.vec_bytes;
-        const bool half_tile = !flat && !use_tuned && !odd_tile && cfg.variant == 0 && cfg.threads == 0 && cfg.unroll == 0 &&
-                               o.group_threads == 0 && mean_vecs > 384 && mean_vecs <= 576;   // (zero-fill tiles may be larger)
-        if (half_tile) {
-            cfg.threads = 256;
-            cfg.unroll = 2;
-            if (cfg.ctas_per_sm == 0) cfg.ctas_per_sm = 3;
         }
         if (cfg.unroll == 0) cfg.unroll = (flat || small) ? 1 : 4;
         if (cfg.threads == 0) cfg.threads = (flat || small) ? 512 : 256;

@@ -116,7 +116,8 @@ copy_tiles_kernel(const CopyParams p)
     const int64_t group_id = GROUPED ? (int64_t)blockIdx.x * groups_per_cta + threadIdx.x / nthr : (int64_t)blockIdx.x;
     const int64_t n_groups = GROUPED ? (int64_t)gridDim.x * groups_per_cta : (int64_t)gridDim.x;
     const uint32_t m_vpr = vpr ? div_magic(vpr) : 0u;
-    const uint32_t tok_vecs = (uint32_t)(hrow / W);   // flat copies: W divides the bytes of a token, not necessarily a row
+    // vectors per token: a flat copy's W divides the bytes of a token, not necessarily a row
+    const uint32_t tok_vecs = flat ? (uint32_t)(hrow / W) : H * vpr;
     const uint32_t m_H = div_magic(H);
 
     // Work items of this group: either every n_groups-th item (the groups sweep the
@@ -178,7 +179,7 @@ copy_tiles_kernel(const CopyParams p)
         const int64_t d_base = t.dst_off + lc * (p.dst.lc_stride >= 0 ? p.dst.lc_stride : buf_lc);
         const bool zero = t.src_off < 0;
         const uint32_t ntok = (uint32_t)t.ntok;
-        const uint32_t nvec = flat ? ntok * tok_vecs : ntok * H * vpr;
+        const uint32_t nvec = ntok * tok_vecs;
         const uint32_t m_inner = head_inner ? m_H : div_magic(ntok);
         const uint32_t inner = head_inner ? H : ntok;
 

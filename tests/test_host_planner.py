@@ -456,7 +456,7 @@ def test_chooser_classes_of_copy():
     pack, unpack, fused = shapes(W.make_config(3, n_req=4, elem_bytes=1))     # 128-byte rows; fused tiles of 16 KiB
     assert (fused["threads"], fused["unroll"], fused["ctas_per_sm"], fused["group_threads"], fused["src_order"]) == (256, 2, 3, 256, 1)
     assert (unpack["threads"], unpack["unroll"], unpack["ctas_per_sm"], unpack["src_order"]) == (256, 4, 2, 0)   # 32 KiB tiles
-    assert (pack["threads"], pack["unroll"], pack["ctas_per_sm"]) == (512, 1, 2)                                 # flat
+    assert (pack["threads"], pack["unroll"], pack["ctas_per_sm"]) == (256, 2, 3)                                 # flat, 16 KiB tiles
     pack, unpack, fused = shapes(W.make_config(4, n_req=2, elem_bytes=1))     # 128-byte rows in full tiles: write order
     assert unpack["src_order"] == 0 and fused["src_order"] == 0 and fused["ctas_per_sm"] == 2
     pack, unpack, fused = shapes(W.make_config(3, n_req=4, num_kv_heads=1))   # 4 KiB tiles: groups of threads
